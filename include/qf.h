@@ -1,0 +1,209 @@
+/*
+ * qf.h -- C ABI of the Q-First cache-side decode-attention library (B200, sm_100a).
+ *
+ * What the library computes (Q-First paper, Section 2 "The device needs only
+ * the query" and Section 5 "The cache may be split anywhere"):
+ *
+ *   The device that holds a request's KV cache receives the query alone, one
+ *   token per request, and sweeps its cached positions.  For a set S of cached
+ *   positions with scores s_i = q.k_i / sqrt(d) and values v_i,
+ *       Z(S) = sum_i e^{s_i},   W(S) = sum_i e^{s_i} v_i,   O(S) = W(S)/Z(S),
+ *   and the device returns (O(S), log Z(S)).  States of disjoint sets merge as
+ *       O(A u B)     = lerp(O(B), O(A), sigma(log Z(A) - log Z(B))),
+ *       log Z(A u B) = logaddexp(log Z(A), log Z(B)),
+ *   with sigma written 1/(1+e^{-x}) so that no magnitude overflows.  An empty
+ *   set is log Z = -inf and a vector that is never read.
+ *
+ * qf_decode_partial computes one such state per (request, KV shard, query
+ * head); qf_combine merges a request's shard states into the full-context
+ * attention output and its log-sum-exp.
+ *
+ * Readings fixed at this boundary where the paper is silent:
+ *   - grouped-query attention: query head h reads KV head h / G, G = Hq/Hkv;
+ *   - the sweep covers cached positions [0, seq_lens[b]) only; the current
+ *     token's own key/value are merged elsewhere (Section 2, the accelerator's
+ *     combine) and are not part of these calls;
+ *   - no causal mask, rotary embedding or normalisation inside the kernels:
+ *     q and the cached keys arrive ready to be multiplied;
+ *   - natural logarithm; the scale multiplies the finished fp32 dot product;
+ *   - o_part is the shard-NORMALISED O(S); m_part is the running maximum
+ *     score (auxiliary: W relative to m is o_part * e^{lse_part - m_part});
+ *   - outputs are fp32; K, V, q are bf16.
+ *
+ * Memory layout (all row-major, all DEVICE memory unless stated):
+ *   q            bf16  [B, Hq, D]
+ *   k_cache,
+ *   v_cache      bf16  [num_pages, Hkv, page_size, D]   (one (page, KV head)
+ *                       block is page_size*D contiguous elements)
+ *   block_table  int32 [B, max_pages_per_req]  logical page -> physical page.
+ *                       May be NULL: then request b's logical page p is
+ *                       physical page b*max_pages_per_req + p.
+ *                       Entries past a request's last page are never read.
+ *   seq_lens     int32 [B]          cached positions of each request
+ *   shard_ranges int32 [B, S, 2]    half-open token range [beg, end) of each
+ *                       shard; clamped to [0, seq_lens[b]]; beg >= end after
+ *                       clamping means an empty shard.  Ranges need not be
+ *                       page-aligned, balanced or disjoint.
+ *   o_part       fp32  [B, S, Hq, D]
+ *   m_part,
+ *   lse_part     fp32  [B, S, Hq]   empty shard: -inf, and o_part = 0
+ *   shard_counts int32 [B]          may be NULL (= S for every request)
+ *   out          fp32  [B, Hq, D];  lse  fp32 [B, Hq]
+ *
+ * Ownership: every pointer is borrowed for the duration of the enqueued work;
+ * the library allocates no device memory, keeps no pointer after the work
+ * completes and has no mutable global state beyond one-time per-device kernel
+ * attributes and a small host-side cache of TMA descriptors keyed by
+ * (pointer, num_pages, num_kv_heads).  `p` is host memory, read before return.
+ *
+ * Asynchrony: every call only enqueues work on `cuda_stream` (a cudaStream_t
+ * passed as void*, NULL = the legacy default stream) and returns without
+ * synchronising, except qf_read_status and qf_decode_step_host, which wait.
+ *
+ * Errors: 0 = success.  A negative return means nothing was enqueued.
+ * Device-side metadata (table entries, ranges) is not validated unless
+ * QF_FLAG_CHECK_BOUNDS is set; with it, an out-of-range page index is skipped
+ * (the tokens of that page contribute nothing), recorded in the workspace
+ * status word and reported by qf_read_status.  No kernel ever traps.
+ */
+#ifndef QF_H_
+#define QF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QF_VERSION 100
+
+enum {
+    QF_OK              = 0,
+    QF_ERR_NULL        = -1, /* a required pointer is NULL                         */
+    QF_ERR_BAD_SHAPE   = -2, /* non-positive size, or Hq not a multiple of Hkv     */
+    QF_ERR_UNSUPPORTED = -3, /* head_dim != 128, page_size != 16, G not in 1,2,4,8 */
+    QF_ERR_WORKSPACE   = -4, /* workspace NULL, misaligned (256 B) or too small    */
+    QF_ERR_CUDA        = -5, /* a CUDA call failed; text via qf_strerror           */
+    QF_ERR_DEVICE      = -6  /* device is not compute capability 10.x             */
+};
+
+enum {
+    QF_FLAG_CHECK_BOUNDS  = 1, /* range-check page indices on the device           */
+    QF_FLAG_SIMPLE_KERNEL = 2  /* use the plain-load sweep kernel (validation aid) */
+};
+
+/* qf_read_status bits */
+enum {
+    QF_STATUS_BAD_PAGE = 1,  /* a block-table entry was outside [0, num_pages)     */
+    QF_STATUS_TIMEOUT  = 2   /* a bounded wait inside a kernel gave up             */
+};
+
+typedef struct qf_params {
+    int32_t batch;             /* B                                              */
+    int32_t num_q_heads;       /* Hq                                             */
+    int32_t num_kv_heads;      /* Hkv                                            */
+    int32_t head_dim;          /* D, must be 128                                 */
+    int32_t page_size;         /* must be 16                                     */
+    int32_t max_pages_per_req; /* row stride of block_table                      */
+    int32_t max_shards;        /* S: row stride of the shard arrays              */
+    int32_t flags;             /* QF_FLAG_*                                      */
+    int64_t num_pages;         /* pages in k_cache / v_cache                     */
+    float   sm_scale;          /* <= 0 means 1/sqrt(head_dim)                    */
+    int32_t reserved;          /* set to 0                                       */
+} qf_params;
+
+/* Library version (QF_VERSION of the build). */
+int qf_version(void);
+
+/* Text for a status code; for QF_ERR_CUDA includes the last CUDA error text.
+ * The pointer is to static/thread-local storage owned by the library. */
+const char *qf_strerror(int status);
+
+/*
+ * Bytes of device scratch qf_decode_partial needs for these parameters
+ * (0 if the parameters are invalid).  The scratch holds the sweep plan
+ * (prefix sums over shards), per-CTA segment states that are merged into the
+ * per-shard states, and a status word.  Contents need not be initialised.
+ * The pointer passed later must be 256-byte aligned.
+ */
+size_t qf_workspace_bytes(const qf_params *p);
+
+/*
+ * Section 2 / Section 5: the cache-side sweep.  For every request b, shard s
+ * and query head h, attends q[b,h,:] over the tokens of shard s (through the
+ * block table, KV head h/G) and writes the shard-normalised output, the
+ * running maximum and the log-sum-exp:
+ *     o_part[b,s,h,:] = O(S),  m_part[b,s,h] = max_i s_i,
+ *     lse_part[b,s,h] = log Z(S).
+ * Every one of the B*S slots is written (empty: 0, -inf, -inf).
+ * All pointers are device pointers; block_table may be NULL (identity).
+ * K/V pool pointers must be 128-byte aligned.  Enqueues on cuda_stream.
+ */
+int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache,
+                      const int32_t *block_table, const int32_t *seq_lens,
+                      const int32_t *shard_ranges,
+                      float *o_part, float *m_part, float *lse_part,
+                      const qf_params *p, void *workspace, size_t workspace_bytes,
+                      void *cuda_stream);
+
+/*
+ * Section 5 merge, n-way: for every (b, h), over shards s < shard_counts[b]
+ * whose lse_part is not -inf,
+ *     M = max_s lse_s,  w_s = e^{lse_s - M},
+ *     out = sum_s w_s o_part_s / sum_s w_s,   lse = M + log sum_s w_s,
+ * which is the pairwise lerp/sigma/logaddexp fold in overflow-safe form.
+ * Vectors of empty shards are never read.  All shards empty: out = 0,
+ * lse = -inf.  All pointers are device pointers; shard_counts may be NULL.
+ */
+int qf_combine(const float *o_part, const float *lse_part, const int32_t *shard_counts,
+               float *out, float *lse,
+               const qf_params *p, void *cuda_stream);
+
+/*
+ * One whole decode step driven from HOST buffers, as a serving loop calls it:
+ * the query and the step's metadata are copied host -> device, the sweep and
+ * the merge run, and the result is copied device -> host.  The KV cache stays
+ * where it lives (that is the protocol: only the query travels).
+ *
+ *   host (pinned for true asynchrony): q_host, seq_lens_host,
+ *       shard_ranges_host, shard_counts_host (may be NULL), out_host, lse_host
+ *   device: k_cache, v_cache, block_table (may be NULL), and `dev_scratch`
+ *       of at least qf_step_scratch_bytes(p) bytes, 256-byte aligned, which
+ *       holds the staged inputs, the shard states, the result and the sweep
+ *       workspace.
+ * Waits for the stream before returning, so out_host/lse_host are valid.
+ */
+size_t qf_step_scratch_bytes(const qf_params *p);
+int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_cache,
+                        const int32_t *block_table, const int32_t *seq_lens_host,
+                        const int32_t *shard_ranges_host, const int32_t *shard_counts_host,
+                        float *out_host, float *lse_host,
+                        const qf_params *p, void *dev_scratch, size_t dev_scratch_bytes,
+                        void *cuda_stream);
+
+/*
+ * Copies the workspace status word (QF_STATUS_* bits, 0 = clean) of the last
+ * qf_decode_partial on this workspace to *host_status.  Synchronises the stream.
+ */
+int qf_read_status(const void *workspace, int32_t *host_status, void *cuda_stream);
+
+/*
+ * Number of kernels the last qf_decode_partial / qf_combine call on this
+ * thread enqueued (for launch accounting in benchmarks).
+ */
+int qf_last_launch_count(void);
+
+/*
+ * Measurement aid (no counterpart in the paper).  While set, every
+ * qf_decode_partial on this thread records `start_event` just before and
+ * `stop_event` just after its sweep kernel on the call's stream, so that a
+ * benchmark can time that one kernel live.  Both are cudaEvent_t handles passed
+ * as void*; pass NULL, NULL to switch it off (the default).
+ */
+int qf_set_profile_events(void *start_event, void *stop_event);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QF_H_ */

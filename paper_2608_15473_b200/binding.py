@@ -1,0 +1,187 @@
+"""Thin ctypes binding over the C ABI in ``include/qf.h``.
+
+Argument marshalling only: every step of the path runs in the CUDA library.
+Functions carry the same names as the C entry points (without the ``qf_``
+prefix).  Tensor arguments may be torch tensors (their ``data_ptr()`` is
+taken), integers (raw addresses) or ``None`` (NULL).
+
+There is no fallback: if ``libqf.so`` has not been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libqf.so"
+
+QF_OK = 0
+QF_ERR_NULL = -1
+QF_ERR_BAD_SHAPE = -2
+QF_ERR_UNSUPPORTED = -3
+QF_ERR_WORKSPACE = -4
+QF_ERR_CUDA = -5
+QF_ERR_DEVICE = -6
+
+QF_FLAG_CHECK_BOUNDS = 1
+QF_FLAG_SIMPLE_KERNEL = 2
+
+QF_STATUS_BAD_PAGE = 1
+QF_STATUS_TIMEOUT = 2
+
+# every symbol include/qf.h declares
+EXPORTS = (
+    "qf_version", "qf_strerror", "qf_workspace_bytes", "qf_decode_partial", "qf_combine",
+    "qf_step_scratch_bytes", "qf_decode_step_host", "qf_read_status", "qf_last_launch_count",
+    "qf_set_profile_events",
+)
+
+
+class QFParams(ctypes.Structure):
+    _fields_ = [
+        ("batch", ctypes.c_int32),
+        ("num_q_heads", ctypes.c_int32),
+        ("num_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32),
+        ("page_size", ctypes.c_int32),
+        ("max_pages_per_req", ctypes.c_int32),
+        ("max_shards", ctypes.c_int32),
+        ("flags", ctypes.c_int32),
+        ("num_pages", ctypes.c_int64),
+        ("sm_scale", ctypes.c_float),
+        ("reserved", ctypes.c_int32),
+    ]
+
+
+class QFError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where} failed with status {status}: {strerror(status)}")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libqf.so (built by ``paper_2608_15473_b200.build``).  Raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2608_15473_b200.build` "
+                "(there is no CPU fallback)")
+        L = ctypes.CDLL(str(LIB_PATH))
+        vp, i32p = ctypes.c_void_p, ctypes.c_void_p
+        pp = ctypes.POINTER(QFParams)
+        L.qf_version.restype = ctypes.c_int
+        L.qf_strerror.restype = ctypes.c_char_p
+        L.qf_strerror.argtypes = [ctypes.c_int]
+        L.qf_workspace_bytes.restype = ctypes.c_size_t
+        L.qf_workspace_bytes.argtypes = [pp]
+        L.qf_step_scratch_bytes.restype = ctypes.c_size_t
+        L.qf_step_scratch_bytes.argtypes = [pp]
+        L.qf_decode_partial.restype = ctypes.c_int
+        L.qf_decode_partial.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, vp, vp, pp, vp, ctypes.c_size_t, vp]
+        L.qf_combine.restype = ctypes.c_int
+        L.qf_combine.argtypes = [vp, vp, i32p, vp, vp, pp, vp]
+        L.qf_decode_step_host.restype = ctypes.c_int
+        L.qf_decode_step_host.argtypes = [vp, vp, vp, i32p, i32p, i32p, i32p, vp, vp, pp, vp, ctypes.c_size_t, vp]
+        L.qf_read_status.restype = ctypes.c_int
+        L.qf_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
+        L.qf_last_launch_count.restype = ctypes.c_int
+        L.qf_set_profile_events.restype = ctypes.c_int
+        L.qf_set_profile_events.argtypes = [vp, vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(x) -> Optional[int]:
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return int(x.data_ptr())
+    if hasattr(x, "ctypes"):  # numpy (host buffers of decode_step_host)
+        return int(x.ctypes.data)
+    raise TypeError(f"cannot take the address of {type(x)}")
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return stream
+    return int(stream.cuda_stream)
+
+
+def params(batch: int, num_q_heads: int, num_kv_heads: int, max_pages_per_req: int, max_shards: int,
+           num_pages: int, head_dim: int = 128, page_size: int = 16, flags: int = 0,
+           sm_scale: float = 0.0) -> QFParams:
+    return QFParams(batch, num_q_heads, num_kv_heads, head_dim, page_size, max_pages_per_req, max_shards,
+                    flags, num_pages, sm_scale, 0)
+
+
+def version() -> int:
+    return int(lib().qf_version())
+
+
+def strerror(status: int) -> str:
+    return lib().qf_strerror(int(status)).decode()
+
+
+def workspace_bytes(p: QFParams) -> int:
+    return int(lib().qf_workspace_bytes(ctypes.byref(p)))
+
+
+def step_scratch_bytes(p: QFParams) -> int:
+    return int(lib().qf_step_scratch_bytes(ctypes.byref(p)))
+
+
+def last_launch_count() -> int:
+    return int(lib().qf_last_launch_count())
+
+
+def set_profile_events(start_event, stop_event) -> None:
+    """cudaEvent_t handles (ints) recorded around the sweep kernel; (None, None) switches it off."""
+    lib().qf_set_profile_events(start_event, stop_event)
+
+
+def decode_partial(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part,
+                   p: QFParams, workspace, workspace_bytes: int, stream=None, check: bool = True) -> int:
+    rc = lib().qf_decode_partial(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table), _ptr(seq_lens),
+                                 _ptr(shard_ranges), _ptr(o_part), _ptr(m_part), _ptr(lse_part),
+                                 ctypes.byref(p), _ptr(workspace), int(workspace_bytes), _stream(stream))
+    if check and rc != QF_OK:
+        raise QFError(rc, "qf_decode_partial")
+    return rc
+
+
+def combine(o_part, lse_part, shard_counts, out, lse, p: QFParams, stream=None, check: bool = True) -> int:
+    rc = lib().qf_combine(_ptr(o_part), _ptr(lse_part), _ptr(shard_counts), _ptr(out), _ptr(lse),
+                          ctypes.byref(p), _stream(stream))
+    if check and rc != QF_OK:
+        raise QFError(rc, "qf_combine")
+    return rc
+
+
+def decode_step_host(q_host, k_cache, v_cache, block_table, seq_lens_host, shard_ranges_host,
+                     shard_counts_host, out_host, lse_host, p: QFParams, dev_scratch, dev_scratch_bytes: int,
+                     stream=None, check: bool = True) -> int:
+    rc = lib().qf_decode_step_host(_ptr(q_host), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
+                                   _ptr(seq_lens_host), _ptr(shard_ranges_host), _ptr(shard_counts_host),
+                                   _ptr(out_host), _ptr(lse_host), ctypes.byref(p), _ptr(dev_scratch),
+                                   int(dev_scratch_bytes), _stream(stream))
+    if check and rc != QF_OK:
+        raise QFError(rc, "qf_decode_step_host")
+    return rc
+
+
+def read_status(workspace, stream=None) -> int:
+    st = ctypes.c_int32(0)
+    rc = lib().qf_read_status(_ptr(workspace), ctypes.byref(st), _stream(stream))
+    if rc != QF_OK:
+        raise QFError(rc, "qf_read_status")
+    return int(st.value)

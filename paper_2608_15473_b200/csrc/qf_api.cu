@@ -1,0 +1,282 @@
+// C ABI of the Q-First decode-attention library: argument validation, workspace
+// carving and kernel launches.  See include/qf.h for the contract.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "../../include/qf.h"
+#include "qf_combine.cuh"
+#include "qf_common.cuh"
+#include "qf_simple.cuh"
+#include "qf_sweep.cuh"
+
+namespace {
+
+thread_local char g_cuda_msg[256] = "";
+thread_local int g_last_launches = 0;
+thread_local cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
+
+int cuda_fail(cudaError_t e, const char *what)
+{
+    std::snprintf(g_cuda_msg, sizeof g_cuda_msg, "%s: %s", what, cudaGetErrorString(e));
+    return QF_ERR_CUDA;
+}
+
+int validate(const qf_params *p)
+{
+    if (!p) return QF_ERR_NULL;
+    if (p->batch <= 0 || p->num_q_heads <= 0 || p->num_kv_heads <= 0 || p->max_pages_per_req <= 0 ||
+        p->max_shards <= 0 || p->num_pages <= 0 || p->head_dim <= 0 || p->page_size <= 0)
+        return QF_ERR_BAD_SHAPE;
+    if (p->num_q_heads % p->num_kv_heads) return QF_ERR_BAD_SHAPE;
+    if (p->head_dim != qf::kHeadDim || p->page_size != qf::kPageSize) return QF_ERR_UNSUPPORTED;
+    const int G = p->num_q_heads / p->num_kv_heads;
+    if (G != 1 && G != 2 && G != 4 && G != 8) return QF_ERR_UNSUPPORTED;
+    // grid dimensions and 32-bit unit counts of the sweep plan
+    if (p->batch > 65535 || p->num_kv_heads > 65535) return QF_ERR_UNSUPPORTED;
+    if ((long long)p->batch * p->max_shards > (1ll << 24)) return QF_ERR_UNSUPPORTED;
+    if ((long long)p->num_pages * p->num_kv_heads * qf::kPageSize >= (1ll << 31)) return QF_ERR_UNSUPPORTED;
+    return QF_OK;
+}
+
+qf::DevParams dev_params(const qf_params *p)
+{
+    qf::DevParams d;
+    d.batch = p->batch;
+    d.num_q_heads = p->num_q_heads;
+    d.num_kv_heads = p->num_kv_heads;
+    d.group = p->num_q_heads / p->num_kv_heads;
+    d.max_pages_per_req = p->max_pages_per_req;
+    d.max_shards = p->max_shards;
+    d.check_bounds = (p->flags & QF_FLAG_CHECK_BOUNDS) ? 1 : 0;
+    d.num_pages = p->num_pages;
+    d.sm_scale = p->sm_scale > 0.f ? p->sm_scale : 1.0f / std::sqrt((float)p->head_dim);
+    return d;
+}
+
+// One-time check per device that this is a compute-capability 10.x part.
+int check_device(int *sm_count)
+{
+    static int cached_major[64];
+    static int cached_sms[64];
+    static bool known[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= 64) return QF_ERR_DEVICE;
+    if (!known[dev]) {
+        int major = 0, sms = 0;
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+        cached_major[dev] = major;
+        cached_sms[dev] = sms;
+        known[dev] = true;
+    }
+    if (cached_major[dev] != 10) return QF_ERR_DEVICE;
+    if (sm_count) *sm_count = cached_sms[dev];
+    return QF_OK;
+}
+
+template <int G>
+int launch_simple(const void *q, const void *k, const void *v, const int32_t *bt, const int32_t *sl,
+                  const int32_t *sr, float *o, float *m, float *l, const qf::DevParams &P, int *status,
+                  cudaStream_t st)
+{
+    dim3 grid(P.max_shards, P.num_kv_heads, P.batch);
+    qf::sweep_simple_kernel<G><<<grid, qf::kSimpleWarps * 32, 0, st>>>(
+        (const uint16_t *)q, (const uint16_t *)k, (const uint16_t *)v, bt, sl, sr, o, m, l, P, status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "sweep_simple_kernel launch");
+    g_last_launches += 1;
+    return QF_OK;
+}
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+}  // namespace
+
+extern "C" {
+
+int qf_version(void) { return QF_VERSION; }
+
+const char *qf_strerror(int status)
+{
+    switch (status) {
+    case QF_OK: return "ok";
+    case QF_ERR_NULL: return "a required pointer is NULL";
+    case QF_ERR_BAD_SHAPE: return "bad shape: sizes must be positive and num_q_heads a multiple of num_kv_heads";
+    case QF_ERR_UNSUPPORTED: return "unsupported: head_dim must be 128, page_size 16, group size 1, 2, 4 or 8";
+    case QF_ERR_WORKSPACE: return "workspace is NULL, not 256-byte aligned, or too small";
+    case QF_ERR_CUDA: return g_cuda_msg[0] ? g_cuda_msg : "CUDA error";
+    case QF_ERR_DEVICE: return "device is not compute capability 10.x (this library is built for sm_100a only)";
+    default: return "unknown status";
+    }
+}
+
+size_t qf_workspace_bytes(const qf_params *p)
+{
+    if (validate(p) != QF_OK) return 0;
+    return qf::workspace_layout(p->batch, p->max_shards, p->num_kv_heads, p->num_q_heads / p->num_kv_heads).total;
+}
+
+int qf_last_launch_count(void) { return g_last_launches; }
+
+int qf_set_profile_events(void *start_event, void *stop_event)
+{
+    g_prof_start = (cudaEvent_t)start_event;
+    g_prof_stop = (cudaEvent_t)stop_event;
+    return QF_OK;
+}
+
+int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache, const int32_t *block_table,
+                      const int32_t *seq_lens, const int32_t *shard_ranges, float *o_part, float *m_part,
+                      float *lse_part, const qf_params *p, void *workspace, size_t workspace_bytes,
+                      void *cuda_stream)
+{
+    g_last_launches = 0;
+    int rc = validate(p);
+    if (rc != QF_OK) return rc;
+    if (!q || !k_cache || !v_cache || !seq_lens || !shard_ranges || !o_part || !m_part || !lse_part)
+        return QF_ERR_NULL;
+    const size_t need = qf_workspace_bytes(p);
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return QF_ERR_WORKSPACE;
+    if (((uintptr_t)k_cache & 127) || ((uintptr_t)v_cache & 127) || ((uintptr_t)q & 15)) return QF_ERR_BAD_SHAPE;
+    int sms = 0;
+    rc = check_device(&sms);
+    if (rc != QF_OK) return rc;
+
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const qf::DevParams P = dev_params(p);
+    const qf::WorkspaceLayout wsl = qf::workspace_layout(P.batch, P.max_shards, P.num_kv_heads, P.group);
+    int *status = reinterpret_cast<int *>((char *)workspace + wsl.header_off);
+
+    if (p->flags & QF_FLAG_SIMPLE_KERNEL) {
+        cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), st);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+        switch (P.group) {
+        case 1: return launch_simple<1>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, status, st);
+        case 2: return launch_simple<2>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, status, st);
+        case 4: return launch_simple<4>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, status, st);
+        default: return launch_simple<8>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, status, st);
+        }
+    }
+
+    int launches = 0;
+    rc = qf::launch_sweep(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P,
+                          (char *)workspace, wsl, sms, st, g_prof_start, g_prof_stop, g_cuda_msg, sizeof g_cuda_msg,
+                          &launches);
+    g_last_launches = launches;
+    return rc;
+}
+
+int qf_combine(const float *o_part, const float *lse_part, const int32_t *shard_counts, float *out, float *lse,
+               const qf_params *p, void *cuda_stream)
+{
+    g_last_launches = 0;
+    int rc = validate(p);
+    if (rc != QF_OK) return rc;
+    if (!o_part || !lse_part || !out || !lse) return QF_ERR_NULL;
+    rc = check_device(nullptr);
+    if (rc != QF_OK) return rc;
+    const long long bh = (long long)p->batch * p->num_q_heads;
+    const unsigned blocks = (unsigned)((bh + qf::kCombineWarps - 1) / qf::kCombineWarps);
+    qf::combine_kernel<<<blocks, qf::kCombineWarps * 32, 0, (cudaStream_t)cuda_stream>>>(
+        o_part, lse_part, shard_counts, out, lse, p->batch, p->num_q_heads, p->max_shards);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "combine_kernel launch");
+    g_last_launches = 1;
+    return QF_OK;
+}
+
+// Carving of the step scratch used by qf_decode_step_host.
+namespace {
+struct StepLayout {
+    size_t q, seq_lens, shard_ranges, shard_counts, o_part, m_part, lse_part, out, lse, workspace, total;
+};
+StepLayout step_layout(const qf_params *p)
+{
+    StepLayout L;
+    const size_t B = p->batch, S = p->max_shards, Hq = p->num_q_heads, D = p->head_dim;
+    size_t off = 0;
+    L.q = off;            off = align256(off + B * Hq * D * 2);
+    L.seq_lens = off;     off = align256(off + B * 4);
+    L.shard_ranges = off; off = align256(off + B * S * 2 * 4);
+    L.shard_counts = off; off = align256(off + B * 4);
+    L.o_part = off;       off = align256(off + B * S * Hq * D * 4);
+    L.m_part = off;       off = align256(off + B * S * Hq * 4);
+    L.lse_part = off;     off = align256(off + B * S * Hq * 4);
+    L.out = off;          off = align256(off + B * Hq * D * 4);
+    L.lse = off;          off = align256(off + B * Hq * 4);
+    L.workspace = off;    off = align256(off + qf_workspace_bytes(p));
+    L.total = off;
+    return L;
+}
+}  // namespace
+
+size_t qf_step_scratch_bytes(const qf_params *p)
+{
+    if (validate(p) != QF_OK) return 0;
+    return step_layout(p).total;
+}
+
+int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_cache, const int32_t *block_table,
+                        const int32_t *seq_lens_host, const int32_t *shard_ranges_host,
+                        const int32_t *shard_counts_host, float *out_host, float *lse_host, const qf_params *p,
+                        void *dev_scratch, size_t dev_scratch_bytes, void *cuda_stream)
+{
+    int rc = validate(p);
+    if (rc != QF_OK) return rc;
+    if (!q_host || !k_cache || !v_cache || !seq_lens_host || !shard_ranges_host || !out_host || !lse_host)
+        return QF_ERR_NULL;
+    const StepLayout L = step_layout(p);
+    if (!dev_scratch || ((uintptr_t)dev_scratch & 255) || dev_scratch_bytes < L.total) return QF_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    char *base = (char *)dev_scratch;
+    const size_t B = p->batch, S = p->max_shards, Hq = p->num_q_heads, D = p->head_dim;
+    cudaError_t e;
+    e = cudaMemcpyAsync(base + L.q, q_host, B * Hq * D * 2, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e, "copy q");
+    e = cudaMemcpyAsync(base + L.seq_lens, seq_lens_host, B * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e, "copy seq_lens");
+    e = cudaMemcpyAsync(base + L.shard_ranges, shard_ranges_host, B * S * 8, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e, "copy shard_ranges");
+    if (shard_counts_host) {
+        e = cudaMemcpyAsync(base + L.shard_counts, shard_counts_host, B * 4, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return cuda_fail(e, "copy shard_counts");
+    }
+    rc = qf_decode_partial(base + L.q, k_cache, v_cache, block_table, (const int32_t *)(base + L.seq_lens),
+                           (const int32_t *)(base + L.shard_ranges), (float *)(base + L.o_part),
+                           (float *)(base + L.m_part), (float *)(base + L.lse_part), p, base + L.workspace,
+                           dev_scratch_bytes - L.workspace, cuda_stream);
+    if (rc != QF_OK) return rc;
+    const int sweep_launches = g_last_launches;
+    rc = qf_combine((const float *)(base + L.o_part), (const float *)(base + L.lse_part),
+                    shard_counts_host ? (const int32_t *)(base + L.shard_counts) : nullptr,
+                    (float *)(base + L.out), (float *)(base + L.lse), p, cuda_stream);
+    if (rc != QF_OK) return rc;
+    g_last_launches += sweep_launches;
+    e = cudaMemcpyAsync(out_host, base + L.out, B * Hq * D * 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "copy out");
+    e = cudaMemcpyAsync(lse_host, base + L.lse, B * Hq * 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "copy lse");
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    return QF_OK;
+}
+
+int qf_read_status(const void *workspace, int32_t *host_status, void *cuda_stream)
+{
+    if (!workspace || !host_status) return QF_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMemcpyAsync(host_status, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync");
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    return QF_OK;
+}
+
+}  // extern "C"

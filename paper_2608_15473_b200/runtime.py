@@ -1,0 +1,106 @@
+"""Device-memory plumbing around the binding: torch owns buffers and streams,
+the CUDA library does all the arithmetic.
+
+``DeviceWorkload`` uploads a host ``Workload`` once and pre-allocates every
+output and the scratch, so that ``sweep()`` / ``merge()`` / ``step()`` only
+enqueue kernels.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as qf
+from .workloads import Workload
+
+
+def _to_dev(a: np.ndarray, device, dtype=None) -> torch.Tensor:
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.view(dtype)
+    return t.to(device, non_blocking=False)
+
+
+class DeviceWorkload:
+    """A workload resident in HBM plus its outputs and scratch."""
+
+    def __init__(self, w: Workload, device="cuda:0", flags: int = 0, identity_table_as_null: bool = False):
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required (there is no CPU path)")
+        self.w = w
+        self.device = torch.device(device)
+        dev = self.device
+        B, Hq, D, S = w.batch, w.num_q_heads, w.head_dim, w.max_shards
+        self.params = qf.params(B, Hq, w.num_kv_heads, w.max_pages_per_req, S, w.num_pages, flags=flags)
+        self.q = _to_dev(w.q.view(np.int16), dev, torch.bfloat16)
+        self.k_cache = _to_dev(w.k_cache.view(np.int16), dev, torch.bfloat16)
+        self.v_cache = _to_dev(w.v_cache.view(np.int16), dev, torch.bfloat16)
+        self.block_table = None if identity_table_as_null else _to_dev(w.block_table, dev)
+        self.seq_lens = _to_dev(w.seq_lens, dev)
+        self.shard_ranges = _to_dev(w.shard_ranges, dev)
+        self.shard_counts = _to_dev(w.shard_counts, dev)
+        self.o_part = torch.empty((B, S, Hq, D), dtype=torch.float32, device=dev)
+        self.m_part = torch.empty((B, S, Hq), dtype=torch.float32, device=dev)
+        self.lse_part = torch.empty((B, S, Hq), dtype=torch.float32, device=dev)
+        self.out = torch.empty((B, Hq, D), dtype=torch.float32, device=dev)
+        self.lse = torch.empty((B, Hq), dtype=torch.float32, device=dev)
+        self.ws_bytes = qf.workspace_bytes(self.params)
+        if self.ws_bytes == 0:
+            raise qf.QFError(qf.QF_ERR_UNSUPPORTED, "qf_workspace_bytes")
+        self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
+        assert self.workspace.data_ptr() % 256 == 0
+
+    def poison_outputs(self) -> None:
+        for t in (self.o_part, self.m_part, self.lse_part, self.out, self.lse):
+            t.fill_(float("nan"))
+
+    def sweep(self, stream=None) -> None:
+        """qf_decode_partial: shard states into o_part / m_part / lse_part."""
+        qf.decode_partial(self.q, self.k_cache, self.v_cache, self.block_table, self.seq_lens,
+                          self.shard_ranges, self.o_part, self.m_part, self.lse_part, self.params,
+                          self.workspace, self.ws_bytes, stream)
+
+    def merge(self, stream=None) -> None:
+        """qf_combine: shard states into out / lse."""
+        qf.combine(self.o_part, self.lse_part, self.shard_counts, self.out, self.lse, self.params, stream)
+
+    def step(self, stream=None) -> int:
+        """One pass of the whole hot path; returns the number of kernels enqueued."""
+        self.sweep(stream)
+        n = qf.last_launch_count()
+        self.merge(stream)
+        return n + qf.last_launch_count()
+
+    def status(self) -> int:
+        return qf.read_status(self.workspace)
+
+    def results(self):
+        """Host copies (float64) of (o_part, m_part, lse_part, out, lse)."""
+        torch.cuda.synchronize(self.device)
+        return tuple(t.detach().cpu().numpy().astype(np.float64)
+                     for t in (self.o_part, self.m_part, self.lse_part, self.out, self.lse))
+
+
+class HostStepper:
+    """End-to-end stepping from pinned host buffers through qf_decode_step_host."""
+
+    def __init__(self, dw: DeviceWorkload):
+        self.dw = dw
+        w = dw.w
+        self.q_host = torch.from_numpy(w.q.view(np.int16).copy()).pin_memory()
+        self.seq_lens_host = torch.from_numpy(w.seq_lens.copy()).pin_memory()
+        self.shard_ranges_host = torch.from_numpy(w.shard_ranges.copy()).pin_memory()
+        self.shard_counts_host = torch.from_numpy(w.shard_counts.copy()).pin_memory()
+        self.out_host = torch.empty((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32).pin_memory()
+        self.lse_host = torch.empty((w.batch, w.num_q_heads), dtype=torch.float32).pin_memory()
+        self.scratch_bytes = qf.step_scratch_bytes(dw.params)
+        self.scratch = torch.empty(self.scratch_bytes, dtype=torch.uint8, device=dw.device)
+        self.h2d_bytes = (self.q_host.numel() * 2 + self.seq_lens_host.numel() * 4 +
+                          self.shard_ranges_host.numel() * 4 + self.shard_counts_host.numel() * 4)
+        self.d2h_bytes = self.out_host.numel() * 4 + self.lse_host.numel() * 4
+
+    def step(self, stream=None) -> None:
+        dw = self.dw
+        qf.decode_step_host(self.q_host, dw.k_cache, dw.v_cache, dw.block_table, self.seq_lens_host,
+                            self.shard_ranges_host, self.shard_counts_host, self.out_host, self.lse_host,
+                            dw.params, self.scratch, self.scratch_bytes, stream)

@@ -1,0 +1,303 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 CPU oracle, element by
+element on the same seeded inputs.  Tolerances: max-abs 2e-3 on outputs, 1e-5 relative on
+log-sum-exp (the contract), plus a much tighter engineering gate (see qf_testlib)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import qf_oracle as orc
+from paper_2608_15473_b200 import binding as qf
+from paper_2608_15473_b200 import build as qf_build
+from paper_2608_15473_b200 import workloads as wl
+from paper_2608_15473_b200.runtime import DeviceWorkload, HostStepper
+
+import qf_testlib as T
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    qf_build.build()
+    assert qf.version() == 100
+
+
+def run(w, flags=0, null_table=False):
+    dw = DeviceWorkload(w, flags=flags, identity_table_as_null=null_table)
+    dw.poison_outputs()
+    dw.step()
+    return dw
+
+
+KERNELS = [pytest.param(0, id="staged"), pytest.param(qf.QF_FLAG_SIMPLE_KERNEL, id="simple")]
+
+
+# T1: every short length, both group sizes, shuffled table: tail-page masking, first-tile guard
+@pytest.mark.parametrize("flags", KERNELS)
+@pytest.mark.parametrize("G", [1, 2, 4, 8])
+def test_every_short_length(G, flags):
+    lens = list(range(1, 49))
+    w = wl.make_workload("t1", lens, [[(0, L)] for L in lens], 2 * G, 2, seed=G, poison_tails=True,
+                         pool_factor=1.3, poison_unused=True)
+    dw = run(w, flags)
+    T.compare_all(dw, w, tag=f"G={G}")
+    assert dw.status() == 0
+
+
+# T2: degenerate and unaligned shard ranges, clamping, L = 0, shard_counts < S
+@pytest.mark.parametrize("flags", KERNELS)
+def test_degenerate_shard_ranges(flags):
+    lens = [100, 0, 37, 300, 16, 1]
+    ranges = [
+        [(0, 7), (7, 7), (7, 33), (33, 100)],
+        [(0, 0), (0, 5), (3, 2), (0, 0)],              # empty request: every shard empty
+        [(0, 500), (-5, 10), (36, 37), (40, 50)],      # clamped at both ends, one fully outside
+        [(0, 128), (128, 129), (129, 257), (257, 300)],
+        [(0, 16), (16, 16), (0, 0), (0, 0)],
+        [(0, 1), (1, 1), (0, 0), (0, 0)],
+    ]
+    counts = [4, 4, 4, 4, 2, 1]
+    w = wl.make_workload("t2", lens, ranges, 8, 2, seed=5, poison_tails=True, shard_counts=counts,
+                         max_pages_per_req=40)
+    dw = run(w, flags)
+    T.compare_all(dw, w)
+    got_op, got_mp, got_lp, got_out, got_lse = dw.results()
+    assert (got_out[1] == 0).all() and np.isneginf(got_lse[1]).all()     # L = 0
+    assert np.isneginf(got_lp[0, 1]).all() and (got_op[0, 1] == 0).all()  # [7,7)
+    assert np.isneginf(got_lp[2, 3]).all()                                # range past the end
+
+
+# T3: a dominant token (logit ~ +22 over the rest) planted at structure boundaries
+@pytest.mark.parametrize("flags", KERNELS)
+@pytest.mark.parametrize("G", [2, 4])
+def test_planted_dominant_token(G, flags):
+    L = 1500
+    shards = [(0, 130), (130, 641), (641, 1024), (1024, 1500)]
+    spots = [0, L - 1, 15, 16, 17, 127, 128, 129, 130, 255, 256, 640, 641, 1023, 1024, 1039, 1040, 1279, 1280, 1499 - 16]
+    B = len(spots)
+    w = wl.make_workload("t3", [L] * B, [shards] * B, 2 * G, 2, seed=11 + G)
+    for b, pos in enumerate(spots):
+        for c in range(2):
+            w.q[b, c * G:(c + 1) * G] = w.q[b, c * G]      # one query per group, so one key dominates all its heads
+            qrow = wl.bf16_bits_to_f32(w.q[b, c * G])
+            w.k_cache[w.block_table[b, pos // 16], c, pos % 16] = wl.f32_to_bf16_bits(2.0 * qrow)
+    dw = run(w, flags)
+    T.compare_all(dw, w, tag=f"G={G}")
+    # the planted token really dominates: out ~ its value row
+    _, _, _, got_out, _ = dw.results()
+    for b, pos in enumerate(spots):
+        v = wl.bf16_bits_to_f64(w.v_cache[w.block_table[b, pos // 16], 0, pos % 16])
+        assert np.abs(got_out[b, 0] - v).max() < 0.05, (b, pos)
+
+
+# T4: NaN poison everywhere the path must not read
+@pytest.mark.parametrize("flags", KERNELS)
+def test_nan_poison_is_never_read(flags):
+    lens = [70, 333, 18]
+    ranges = [[(5, 40), (40, 70)], [(3, 200), (200, 321)], [(1, 2), (2, 17)]]
+    w = wl.make_workload("t4", lens, ranges, 8, 2, seed=13, pool_factor=2.0, poison_unused=True, poison_tails=True)
+    nan = np.uint16(0x7FC0)
+    for b, rr in enumerate(ranges):  # poison the tokens outside every shard range too
+        covered = np.zeros(lens[b], bool)
+        for lo, hi in rr:
+            covered[lo:hi] = True
+        for i in np.nonzero(~covered)[0]:
+            w.k_cache[w.block_table[b, i // 16], :, i % 16] = nan
+            w.v_cache[w.block_table[b, i // 16], :, i % 16] = nan
+    dw = run(w, flags)
+    errs = T.compare_all(dw, w)
+    assert errs["out"] < T.ENG_OUT
+    # empty shards' vectors are never read by the combine
+    w2 = wl.make_workload("t4b", [64], [[(0, 30), (30, 30), (30, 64)]], 4, 2, seed=14)
+    dw2 = DeviceWorkload(w2, flags=flags)
+    dw2.sweep()
+    dw2.o_part[0, 1].fill_(float("nan"))
+    dw2.merge()
+    got = dw2.results()
+    ref = T.oracle_all(w2)
+    assert T.out_err(got[3], ref[3]) < T.ENG_OUT and T.lse_err(got[4], ref[4]) < T.ENG_LSE
+
+
+# T5: the same logical data under two page permutations gives bit-identical results
+def test_paging_invariance_bitwise():
+    lens = [257, 1000, 31]
+    ranges = [wl.even_shards(L, 3) for L in lens]
+    a = wl.make_workload("t5", lens, ranges, 8, 2, seed=17, table="identity")
+    rng = np.random.default_rng(3)
+    P = 200
+    perm = rng.permutation(P)
+    npg = [(L + 15) // 16 for L in lens]
+    bt = np.full((3, a.max_pages_per_req), -1, np.int32)
+    kc = np.full((P, 2, 16, 128), 0x7FC0, np.uint16)
+    vc = np.full((P, 2, 16, 128), 0x7FC0, np.uint16)
+    pos = 0
+    for b in range(3):
+        for p in range(npg[b]):
+            bt[b, p] = perm[pos]
+            kc[perm[pos]] = a.k_cache[a.block_table[b, p]]
+            vc[perm[pos]] = a.v_cache[a.block_table[b, p]]
+            pos += 1
+    b_ = wl.Workload("t5b", a.batch, a.num_q_heads, a.num_kv_heads, a.max_pages_per_req, a.max_shards, P,
+                     a.q, kc, vc, bt, a.seq_lens, a.shard_ranges, a.shard_counts)
+    ra = run(a).results()
+    rb = run(b_).results()
+    rc = run(a, null_table=True).results()   # NULL block table = identity
+    for x, y, z in zip(ra, rb, rc):
+        assert np.array_equal(x, y) and np.array_equal(x, z)
+    T.compare_all(run(a), a)
+
+
+# T6: extremes: logits near +85, near -85, mixed across shards
+@pytest.mark.parametrize("flags", KERNELS)
+def test_extreme_logits(flags):
+    L = 2048
+    w = wl.make_workload("t6", [L] * 3, [wl.even_shards(L, 4)] * 3, 4, 2, seed=19, table="shuffled")
+    G = 2
+    for c in range(2):
+        for b in range(3):
+            w.q[b, c * G:(c + 1) * G] = w.q[b, c * G]
+    def set_logit(b, toks, target):
+        for c in range(2):
+            qv = wl.bf16_bits_to_f64(w.q[b, c * G])
+            k = qv * (target * np.sqrt(128.0) / (qv @ qv))
+            for i in toks:
+                w.k_cache[w.block_table[b, i // 16], c, i % 16] = wl.f32_to_bf16_bits(k.astype(np.float32))
+    set_logit(0, range(L), 85.0)                    # everything near +85: naive sum of e^s overflows fp32
+    set_logit(1, range(L), -85.0)                   # everything near -85: naive sum underflows to 0
+    set_logit(2, range(0, 512), 85.0)               # shard 0 at +85, shard 3 at -85
+    set_logit(2, range(1536, L), -85.0)
+    dw = run(w, flags)
+    T.compare_all(dw, w)
+    _, _, got_lp, _, got_lse = dw.results()
+    assert abs(got_lse[0, 0] - (85 + np.log(L))) < 0.5 and abs(got_lse[1, 0] - (-85 + np.log(L))) < 0.5
+    assert got_lp[2, 0, 0] > 80 and got_lp[2, 3, 0] < -70
+
+
+# T7: the combine alone on hand-made shard states
+def test_combine_on_handmade_states():
+    rng = np.random.default_rng(23)
+    cases = [(100.0, 100.0), (85.0, 91.0), (90.0, -90.0), (-90.0, 90.0), (3.0, -np.inf), (-np.inf, 3.0),
+             (-np.inf, -np.inf), (0.0, 0.0), (-0.5, 0.25), (88.0, 89.5)]
+    B, S, Hq, D = len(cases), 2, 4, 128
+    o = rng.standard_normal((B, S, Hq, D)).astype(np.float32)
+    l = np.zeros((B, S, Hq), np.float32)
+    for b, (a, c) in enumerate(cases):
+        l[b, 0], l[b, 1] = a, c
+    o[np.isneginf(l)] = np.nan   # empty shards hold garbage that must not be read
+    sh = orc.Shape(batch=B, num_q_heads=Hq, num_kv_heads=2, max_shards=S)
+    p = qf.params(B, Hq, 2, 4, S, 4)
+    for order in ([0, 1], [1, 0]):
+        oo, ll = o[:, order].copy(), l[:, order].copy()
+        ref_out, ref_lse = orc.combine(oo.astype(np.float64), ll.astype(np.float64), None, sh)
+        fold_out, fold_lse = orc.combine_fold(oo.astype(np.float64), ll.astype(np.float64), None, sh)
+        d_o, d_l = torch.from_numpy(oo).cuda(), torch.from_numpy(ll).cuda()
+        out = torch.full((B, Hq, D), float("nan"), device="cuda")
+        lse = torch.full((B, Hq), float("nan"), device="cuda")
+        qf.combine(d_o, d_l, None, out, lse, p)
+        torch.cuda.synchronize()
+        assert T.out_err(out.cpu().numpy(), ref_out) < 1e-6
+        assert T.lse_err(lse.cpu().numpy(), ref_lse) < 1e-6
+        assert T.out_err(out.cpu().numpy(), fold_out) < 1e-6 and T.lse_err(lse.cpu().numpy(), fold_lse) < 1e-6
+    # shard_counts: slots past the count are ignored even if finite
+    cnt = torch.ones(B, dtype=torch.int32, device="cuda")
+    d_o, d_l = torch.from_numpy(o).cuda(), torch.from_numpy(l).cuda()
+    out = torch.empty((B, Hq, D), device="cuda")
+    lse = torch.empty((B, Hq), device="cuda")
+    qf.combine(d_o, d_l, cnt, out, lse, p)
+    ref_out, ref_lse = orc.combine(o.astype(np.float64), l.astype(np.float64), np.ones(B, np.int32), sh)
+    assert T.out_err(out.cpu().numpy(), ref_out) < 1e-6 and T.lse_err(lse.cpu().numpy(), ref_lse) < 1e-6
+
+
+# medium cases that span many stages, several CTA slices and ragged tails
+@pytest.mark.parametrize("flags", KERNELS)
+@pytest.mark.parametrize("G,seed", [(2, 0), (4, 1), (8, 2), (1, 3)])
+def test_medium_ragged_batch(G, seed, flags):
+    rng = np.random.default_rng(seed)
+    lens = rng.integers(1, 6000, size=12).tolist() + [4096, 129, 127]
+    ranges = [wl.fixed_shards(L, 1000) for L in lens]
+    w = wl.make_workload("med", lens, ranges, 2 * G, 2, seed=seed, pool_factor=1.2, poison_unused=True,
+                         poison_tails=True)
+    dw = run(w, flags)
+    T.compare_all(dw, w, tag=f"G={G}")
+    assert dw.status() == 0
+
+
+def test_long_single_request_many_segments():
+    # one request whose single shard is split over every SM by the balanced schedule
+    L = 150_001
+    w = wl.make_workload("long", [L], [[(0, L)]], 4, 2, seed=29)
+    dw = run(w)
+    T.compare_all(dw, w)
+
+
+def test_small_configs_elementwise():
+    for w in (wl.config1(seed=0), wl.config2(seed=1, batch=6), wl.config3(seed=2, batch=4, hi=9000),
+              wl.config4(seed=0, ctx=1 << 15, n_shards=16, n_plant=400),
+              wl.config5(seed=0, batch=12, hi=8192)):
+        dw = run(w)
+        T.compare_all(dw, w, tag=w.name)
+        dws = run(w, qf.QF_FLAG_SIMPLE_KERNEL)
+        T.compare_all(dws, w, tag=w.name + "/simple")
+
+
+# T9: run-to-run determinism and canaries around the outputs
+def test_determinism_and_no_stray_writes():
+    w = wl.config3(seed=5, batch=6, hi=12000)
+    dw = DeviceWorkload(w)
+    canary = 1234.5
+    bufs = {}
+    for name in ("o_part", "m_part", "lse_part", "out", "lse"):
+        t = getattr(dw, name)
+        big = torch.full((t.numel() + 512,), canary, dtype=torch.float32, device="cuda")
+        setattr(dw, name, big[256:256 + t.numel()].view(t.shape))
+        bufs[name] = big
+    runs = []
+    for _ in range(3):
+        dw.poison_outputs()
+        dw.step()
+        runs.append([r.copy() for r in dw.results()])
+    for r in runs[1:]:
+        for x, y in zip(runs[0], r):
+            assert np.array_equal(x, y)
+    for name, big in bufs.items():
+        assert (big[:256] == canary).all() and (big[-256:] == canary).all(), name
+    T.compare_all(dw, w)
+
+
+# debug flag: an out-of-range page index is skipped and reported, never a fault
+@pytest.mark.parametrize("flags", KERNELS)
+def test_bad_page_index_is_reported_not_followed(flags):
+    L = 400
+    w = wl.make_workload("bad", [L, L], [[(0, L)], [(0, L)]], 4, 2, seed=31)
+    good_entry = int(w.block_table[1, 3])
+    w.block_table[1, 3] = w.num_pages + 7
+    dw = run(w, flags | qf.QF_FLAG_CHECK_BOUNDS)
+    assert dw.status() & qf.QF_STATUS_BAD_PAGE
+    # request 0 is untouched; request 1 equals the sweep with page 3's tokens left out
+    w.block_table[1, 3] = good_entry
+    w2 = wl.make_workload("bad", [L, L], [[(0, L)], [(0, 48), (64, L)]], 4, 2, seed=31)
+    ref = T.oracle_all(w2)
+    got = dw.results()
+    assert T.out_err(got[3][0], ref[3][0]) < T.ENG_OUT
+    assert T.out_err(got[3][1], ref[3][1]) < T.ENG_OUT and T.lse_err(got[4][1], ref[4][1]) < T.ENG_LSE
+
+
+def test_host_step_matches_device_path():
+    w = wl.config3(seed=7, batch=5, hi=6000)
+    dw = run(w)
+    hs = HostStepper(dw)
+    hs.step()
+    _, _, _, out, lse = dw.results()
+    assert np.array_equal(hs.out_host.numpy().astype(np.float64), out)
+    assert np.array_equal(hs.lse_host.numpy().astype(np.float64), lse)
+    assert hs.h2d_bytes > 0 and hs.d2h_bytes == out.size * 4 + lse.size * 4
+
+
+# T8: the benchmark configurations at full size, sampled outputs
+@pytest.mark.parametrize("cfg", [2, 3, 4])
+def test_full_size_configs_sampled(cfg):
+    w = wl.CONFIGS[cfg](seed=0)
+    dw = run(w)
+    errs = T.compare_sampled(dw, w, seed=cfg, tag=w.name)
+    print(w.name, errs)
+    assert dw.status() == 0
