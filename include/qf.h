@@ -85,7 +85,8 @@ enum {
     QF_ERR_UNSUPPORTED = -3, /* head_dim != 128, page_size != 16, G not in 1,2,4,8 */
     QF_ERR_WORKSPACE   = -4, /* workspace NULL, misaligned (256 B) or too small    */
     QF_ERR_CUDA        = -5, /* a CUDA call failed; text via qf_strerror           */
-    QF_ERR_DEVICE      = -6  /* device is not compute capability 10.x             */
+    QF_ERR_DEVICE      = -6, /* device is not compute capability 10.x             */
+    QF_ERR_STATIC_SCRATCH = -7 /* problem too large for qf_decode_partial_static   */
 };
 
 enum {
@@ -202,6 +203,49 @@ int qf_last_launch_count(void);
  * as void*; pass NULL, NULL to switch it off (the default).
  */
 int qf_set_profile_events(void *start_event, void *stop_event);
+
+/*
+ * The sweep for callers that cannot allocate.  (The paper has no counterpart:
+ * this entry point exists for the library's users, not for the method.)
+ *
+ * qf_decode_partial asks its caller for a scratch buffer.  Some callers have no
+ * way to get one on the decode path: their device memory was partitioned at
+ * start-up and the pool is closed, or they sit inside a framework operator that
+ * is handed its input and output tensors and nothing else, or they run at a
+ * point where calling cudaMalloc is off limits because it may block on, or
+ * synchronise, the whole device.  This variant takes the same inputs and
+ * outputs and no workspace: it uses a fixed array of QF_STATIC_SCRATCH_BYTES
+ * that is part of the library's device image (so every GPU that loads the
+ * library carries those bytes until the process ends).  It calls no cudaMalloc,
+ * cudaFree or any routine that allocates.
+ *
+ * Limits and rules:
+ *   - if qf_workspace_bytes(p) exceeds QF_STATIC_SCRATCH_BYTES the call returns
+ *     QF_ERR_STATIC_SCRATCH and enqueues nothing; qf_static_scratch_error()
+ *     then says how many bytes were needed.  Roughly, batch * max_shards *
+ *     num_kv_heads may reach about 3,400 at a group size of 4.
+ *   - the first call on each device looks the array's device address up
+ *     (cudaGetSymbolAddress, with that device current) and remembers it; make
+ *     that first call before starting any stream capture.
+ *   - all calls on a device share the one array, which keeps whatever the last
+ *     call left in it.  Each call rewrites everything it later reads (status
+ *     word, plan, segment states), so back-to-back calls on one stream are
+ *     safe; two calls whose kernels may overlap on the GPU (different streams,
+ *     no ordering between them) race on the array and must not be issued.
+ *   - qf_read_status cannot be pointed at the array from outside; use
+ *     qf_decode_partial with QF_FLAG_CHECK_BOUNDS when a status is wanted.
+ * Everything else (arguments, layouts, results, error codes, asynchrony) is as
+ * for qf_decode_partial.
+ */
+#define QF_STATIC_SCRATCH_BYTES (8u << 20)
+int qf_decode_partial_static(const void *q, const void *k_cache, const void *v_cache,
+                             const int32_t *block_table, const int32_t *seq_lens,
+                             const int32_t *shard_ranges,
+                             float *o_part, float *m_part, float *lse_part,
+                             const qf_params *p, void *cuda_stream);
+
+/* Text describing the last QF_ERR_STATIC_SCRATCH / set-up failure on this thread. */
+const char *qf_static_scratch_error(void);
 
 #ifdef __cplusplus
 }

@@ -23,6 +23,8 @@ QF_ERR_UNSUPPORTED = -3
 QF_ERR_WORKSPACE = -4
 QF_ERR_CUDA = -5
 QF_ERR_DEVICE = -6
+QF_ERR_STATIC_SCRATCH = -7
+QF_STATIC_SCRATCH_BYTES = 8 << 20
 
 QF_FLAG_CHECK_BOUNDS = 1
 QF_FLAG_SIMPLE_KERNEL = 2
@@ -34,7 +36,7 @@ QF_STATUS_TIMEOUT = 2
 EXPORTS = (
     "qf_version", "qf_strerror", "qf_workspace_bytes", "qf_decode_partial", "qf_combine",
     "qf_step_scratch_bytes", "qf_decode_step_host", "qf_read_status", "qf_last_launch_count",
-    "qf_set_profile_events",
+    "qf_set_profile_events", "qf_decode_partial_static", "qf_static_scratch_error",
 )
 
 
@@ -92,6 +94,9 @@ def lib() -> ctypes.CDLL:
         L.qf_last_launch_count.restype = ctypes.c_int
         L.qf_set_profile_events.restype = ctypes.c_int
         L.qf_set_profile_events.argtypes = [vp, vp]
+        L.qf_decode_partial_static.restype = ctypes.c_int
+        L.qf_decode_partial_static.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, vp, vp, pp, vp]
+        L.qf_static_scratch_error.restype = ctypes.c_char_p
         _lib = L
     return _lib
 
@@ -156,6 +161,18 @@ def decode_partial(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_p
                                  ctypes.byref(p), _ptr(workspace), int(workspace_bytes), _stream(stream))
     if check and rc != QF_OK:
         raise QFError(rc, "qf_decode_partial")
+    return rc
+
+
+def decode_partial_static(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part,
+                          p: QFParams, stream=None, check: bool = True) -> int:
+    """The sweep with the library's built-in scratch array: for callers that cannot allocate."""
+    rc = lib().qf_decode_partial_static(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
+                                        _ptr(seq_lens), _ptr(shard_ranges), _ptr(o_part), _ptr(m_part),
+                                        _ptr(lse_part), ctypes.byref(p), _stream(stream))
+    if check and rc != QF_OK:
+        detail = lib().qf_static_scratch_error().decode()
+        raise QFError(rc, "qf_decode_partial_static" + (f" ({detail})" if detail else ""))
     return rc
 
 

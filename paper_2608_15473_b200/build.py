@@ -9,7 +9,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libqf.so"
-SOURCES = [CSRC / "qf_api.cu"]
+SOURCES = [CSRC / "qf_api.cu", CSRC / "qf_static_scratch.cu"]
 HEADERS = sorted(CSRC.glob("*.cuh")) + [PKG.parent / "include" / "qf.h"]
 
 NVCC_FLAGS = [

@@ -113,6 +113,7 @@ const char *qf_strerror(int status)
     case QF_ERR_WORKSPACE: return "workspace is NULL, not 256-byte aligned, or too small";
     case QF_ERR_CUDA: return g_cuda_msg[0] ? g_cuda_msg : "CUDA error";
     case QF_ERR_DEVICE: return "device is not compute capability 10.x (this library is built for sm_100a only)";
+    case QF_ERR_STATIC_SCRATCH: return "problem needs more scratch than the built-in static array; use qf_decode_partial";
     default: return "unknown status";
     }
 }
