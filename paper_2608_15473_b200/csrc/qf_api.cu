@@ -36,7 +36,7 @@ int validate(const qf_params *p)
     if (G != 1 && G != 2 && G != 4 && G != 8) return QF_ERR_UNSUPPORTED;
     // grid dimensions and 32-bit unit counts of the sweep plan
     if (p->batch > 65535 || p->num_kv_heads > 65535) return QF_ERR_UNSUPPORTED;
-    if ((long long)p->batch * p->max_shards > (1ll << 24)) return QF_ERR_UNSUPPORTED;
+    if ((long long)p->batch * p->max_shards * p->num_kv_heads > (1ll << 22)) return QF_ERR_UNSUPPORTED;
     if ((long long)p->num_pages * p->num_kv_heads * qf::kPageSize >= (1ll << 31)) return QF_ERR_UNSUPPORTED;
     return QF_OK;
 }
@@ -83,12 +83,12 @@ int check_device(int *sm_count)
 
 template <int G>
 int launch_simple(const void *q, const void *k, const void *v, const int32_t *bt, const int32_t *sl,
-                  const int32_t *sr, float *o, float *m, float *l, const qf::DevParams &P, int *status,
-                  cudaStream_t st)
+                  const int32_t *sr, float *o, float *m, float *l, const qf::DevParams &P,
+                  unsigned long long *header, unsigned long long epoch, cudaStream_t st)
 {
     dim3 grid(P.max_shards, P.num_kv_heads, P.batch);
     qf::sweep_simple_kernel<G><<<grid, qf::kSimpleWarps * 32, 0, st>>>(
-        (const uint16_t *)q, (const uint16_t *)k, (const uint16_t *)v, bt, sl, sr, o, m, l, P, status);
+        (const uint16_t *)q, (const uint16_t *)k, (const uint16_t *)v, bt, sl, sr, o, m, l, P, header, epoch);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "sweep_simple_kernel launch");
     g_last_launches += 1;
@@ -153,23 +153,22 @@ int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache, c
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const qf::DevParams P = dev_params(p);
     const qf::WorkspaceLayout wsl = qf::workspace_layout(P.batch, P.max_shards, P.num_kv_heads, P.group);
-    int *status = reinterpret_cast<int *>((char *)workspace + wsl.header_off);
+    unsigned long long *header = reinterpret_cast<unsigned long long *>((char *)workspace + wsl.header_off);
+    const unsigned long long epoch = qf::next_epoch();
 
     if (p->flags & QF_FLAG_SIMPLE_KERNEL) {
-        cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), st);
-        if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
         switch (P.group) {
-        case 1: return launch_simple<1>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, status, st);
-        case 2: return launch_simple<2>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, status, st);
-        case 4: return launch_simple<4>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, status, st);
-        default: return launch_simple<8>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, status, st);
+        case 1: return launch_simple<1>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, header, epoch, st);
+        case 2: return launch_simple<2>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, header, epoch, st);
+        case 4: return launch_simple<4>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, header, epoch, st);
+        default: return launch_simple<8>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, header, epoch, st);
         }
     }
 
     int launches = 0;
     rc = qf::launch_sweep(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P,
-                          (char *)workspace, wsl, sms, st, g_prof_start, g_prof_stop, g_cuda_msg, sizeof g_cuda_msg,
-                          &launches);
+                          (char *)workspace, wsl, sms, epoch, st, g_prof_start, g_prof_stop, g_cuda_msg,
+                          sizeof g_cuda_msg, &launches);
     g_last_launches = launches;
     return rc;
 }
@@ -273,10 +272,14 @@ int qf_read_status(const void *workspace, int32_t *host_status, void *cuda_strea
 {
     if (!workspace || !host_status) return QF_ERR_NULL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    cudaError_t e = cudaMemcpyAsync(host_status, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+    // word 0: status bits tagged with the epoch of the launch that set them; word 1: epoch of the last launch
+    unsigned long long words[2] = {0, 0};
+    cudaError_t e = cudaMemcpyAsync(words, workspace, sizeof words, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync");
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    const bool current = (words[0] >> qf::kEpochShift) == words[1];
+    *host_status = current ? (int32_t)(words[0] & qf::kEpochLowMask) : 0;
     return QF_OK;
 }
 

@@ -1,6 +1,7 @@
 // Merge of shard states (Section 5): n-way, overflow-safe form of the pairwise
 // lerp / sigma / logaddexp combine.  One warp per (request, query head); each
-// lane owns four channels, so a shard's 512-byte vector is one coalesced read.
+// lane owns four channels, so a shard's 512-byte vector is one coalesced read.  A slot whose
+// log Z is -inf contributes through a select, never a multiply, so garbage in it is harmless.
 #pragma once
 
 #include "qf_common.cuh"
@@ -31,18 +32,38 @@ combine_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_p
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float wsum = 0.f;
     if (M != neg_inf()) {
-        for (int s = 0; s < ns; ++s) {
-            const float ls = lrow[(size_t)s * num_q_heads];
-            if (ls == neg_inf()) continue;          // empty shard: vector never read
-            const float w = expf(ls - M);           // in (0, 1]: cannot overflow
-            const float4 o = *reinterpret_cast<const float4 *>(
-                o_part + (((size_t)b * max_shards + s) * num_q_heads + h) * kHeadDim + lane * 4);
+        const float *obase = o_part + (((size_t)b * max_shards) * num_q_heads + h) * kHeadDim + lane * 4;
+        const size_t ostride = (size_t)num_q_heads * kHeadDim;
+        for (int base = 0; base < ns; base += 32) {
+            // lane s holds shard (base+s)'s weight e^{lse_s - M}: in (0, 1], cannot overflow; 0 for empty shards
+            const int sl = base + lane;
+            const float ls = (sl < ns) ? lrow[(size_t)sl * num_q_heads] : neg_inf();
+            const float w = (ls == neg_inf()) ? 0.f : expf(ls - M);
             wsum += w;
-            acc.x = fmaf(w, o.x, acc.x);
-            acc.y = fmaf(w, o.y, acc.y);
-            acc.z = fmaf(w, o.z, acc.z);
-            acc.w = fmaf(w, o.w, acc.w);
+            const int cnt = min(32, ns - base);
+            for (int j = 0; j < cnt; j += 4) {
+                float wj[4];
+                float4 o[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {   // four independent 512-byte reads in flight
+                    wj[u] = __shfl_sync(0xffffffffu, w, (j + u) & 31);
+                    if (j + u >= cnt) wj[u] = 0.f;
+                    o[u] = (j + u < cnt) ? *reinterpret_cast<const float4 *>(obase + (size_t)(base + j + u) * ostride)
+                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (wj[u] != 0.f) {         // an empty shard's vector is loaded but never used
+                        acc.x = fmaf(wj[u], o[u].x, acc.x);
+                        acc.y = fmaf(wj[u], o[u].y, acc.y);
+                        acc.z = fmaf(wj[u], o[u].z, acc.z);
+                        acc.w = fmaf(wj[u], o[u].w, acc.w);
+                    }
+                }
+            }
         }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, off);
         const float inv = 1.f / wsum;
         acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
     }

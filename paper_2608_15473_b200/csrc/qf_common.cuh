@@ -34,6 +34,42 @@ __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000u);
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi_to_f32(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
+// The workspace is never assumed to be initialised.  Words that must "start at zero" for a launch
+// (the status word, the per-unit arrival counters) carry the launch's epoch in their upper 54 bits:
+// a word whose epoch differs from the current launch's counts as zero.
+constexpr int kEpochShift = 10;
+constexpr unsigned long long kEpochLowMask = (1ull << kEpochShift) - 1;
+
+// Header words (unsigned long long) at the start of the workspace.
+enum { kHdrStatus = 0, kHdrLastEpoch = 1, kHdrTotals = 2 /* low: total units, high: units per CTA */ };
+
+// OR `bits` into an epoch-tagged word.  Bounded retry; contention is at most a few writers.
+__device__ __forceinline__ void epoch_or(unsigned long long *w, unsigned long long epoch, unsigned bits)
+{
+    unsigned long long old = *reinterpret_cast<volatile unsigned long long *>(w);
+    for (int tries = 0; tries < (1 << 16); ++tries) {
+        const unsigned long long cur = ((old >> kEpochShift) == epoch) ? (old & kEpochLowMask) : 0ull;
+        const unsigned long long neu = (epoch << kEpochShift) | cur | bits;
+        const unsigned long long prev = atomicCAS(w, old, neu);
+        if (prev == old) return;
+        old = prev;
+    }
+}
+
+// Add one to an epoch-tagged counter and return the new count (0 if the bounded retry ran out).
+__device__ __forceinline__ unsigned epoch_arrive(unsigned long long *w, unsigned long long epoch)
+{
+    unsigned long long old = *reinterpret_cast<volatile unsigned long long *>(w);
+    for (int tries = 0; tries < (1 << 16); ++tries) {
+        const unsigned long long cur = ((old >> kEpochShift) == epoch) ? (old & kEpochLowMask) : 0ull;
+        const unsigned long long neu = (epoch << kEpochShift) | (cur + 1);
+        const unsigned long long prev = atomicCAS(w, old, neu);
+        if (prev == old) return (unsigned)(cur + 1);
+        old = prev;
+    }
+    return 0;
+}
+
 // Clamp a shard's token range to the request's cached length.
 __device__ __forceinline__ void clamp_range(int r0, int r1, int len, int &beg, int &end)
 {

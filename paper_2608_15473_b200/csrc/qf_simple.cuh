@@ -16,11 +16,13 @@ sweep_simple_kernel(const uint16_t *__restrict__ q, const uint16_t *__restrict__
                     const uint16_t *__restrict__ v_cache, const int *__restrict__ block_table,
                     const int *__restrict__ seq_lens, const int *__restrict__ shard_ranges,
                     float *__restrict__ o_part, float *__restrict__ m_part, float *__restrict__ lse_part,
-                    DevParams P, int *status)
+                    DevParams P, unsigned long long *header, unsigned long long epoch)
 {
     const int s = blockIdx.x, c = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = P.max_shards, Hq = P.num_q_heads, Hkv = P.num_kv_heads;
+
+    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) header[kHdrLastEpoch] = epoch;
 
     int beg, end;
     clamp_range(shard_ranges[(b * S + s) * 2], shard_ranges[(b * S + s) * 2 + 1], seq_lens[b], beg, end);
@@ -46,7 +48,7 @@ sweep_simple_kernel(const uint16_t *__restrict__ q, const uint16_t *__restrict__
         long long phys = block_table ? (long long)block_table[(size_t)b * P.max_pages_per_req + lp]
                                      : (long long)b * P.max_pages_per_req + lp;
         if (P.check_bounds && (phys < 0 || phys >= P.num_pages)) {
-            if (lane == 0) atomicOr(status, kStatusBadPage);
+            if (lane == 0) epoch_or(header + kHdrStatus, epoch, kStatusBadPage);
             continue;
         }
         const size_t row = (((size_t)phys * Hkv + c) * kPageSize + slot) * kHeadDim + lane * 4;

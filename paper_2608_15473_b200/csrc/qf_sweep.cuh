@@ -1,52 +1,64 @@
-// The staged sweep: plan -> persistent TMA/tensor-core sweep -> segment merge.
+// The staged sweep: one persistent kernel that plans, streams and merges.
 //
 // Section 5 of the Q-First paper lets a cache be split anywhere: partial states
 // (W, Z) add over disjoint token sets.  The user-visible split is the shard; this
-// file splits further, invisibly, so that every SM streams the same number of KV
-// bytes whatever the batch looks like:
+// kernel splits further, invisibly, so that every SM streams the same number of KV
+// bytes whatever the batch looks like.
 //
-//   plan_kernel   turns (seq_lens, shard_ranges) into a prefix sum over
-//                 "stage units" (8 pages = 128 tokens of one KV head of one shard);
-//   sweep_kernel  one persistent CTA per SM takes an equal contiguous slice of the
-//                 unit space.  A producer warp walks the slice, looks pages up in
-//                 the block table and issues TMA tile loads (128B-swizzled) into a
-//                 3-stage shared-memory ring; 8 consumer warps each take one page of
-//                 a stage: S = K Q^T on tensor cores (tokens on M, the group's heads
-//                 on N), fp32 online softmax, P split into bf16 hi+lo, O^T += V^T P^T.
-//                 A slice boundary inside a shard yields a segment state in scratch;
-//   merge_kernel  merges the segments of a (shard, KV head) into o_part/m_part/
-//                 lse_part, and writes the empty-shard convention.
+//   plan      every CTA turns (seq_lens, shard_ranges) into a prefix sum over "stage
+//             units" (8 pages = 128 tokens of one KV head of one shard) in shared
+//             memory and takes an equal contiguous slice of the unit space (no atomics,
+//             no work queue).  Batches with more than kMaxSmemEntries (request, shard)
+//             pairs use a separate plan kernel that leaves the prefix in scratch.
+//   stream    a producer warp walks the slice, looks pages up in the block table and
+//             issues one 4 KB TMA box per K or V page (128B-swizzled) into a 3-stage shared-memory ring;
+//             8 consumer warps each take one page of a stage: S = K Q^T on tensor cores
+//             (tokens on M, the group's heads on N), fp32 online softmax, P split into
+//             bf16 hi+lo, O^T += V^T P^T.
+//   merge     a slice boundary inside a (shard, KV head) unit leaves segment states in
+//             scratch; the last CTA to finish a segment of that unit (epoch-tagged
+//             arrival counter) merges them in fixed order into o_part/m_part/lse_part.
+//             Empty shards get (0, -inf, -inf) from the consumer warps' prologue.
 //
 // All waits are bounded: a wait that runs out sets QF_STATUS_TIMEOUT, raises a
-// CTA-wide abort flag and every warp leaves through the same exit.
+// CTA-wide abort flag and every warp leaves.  No CTA ever waits for another CTA.
 #pragma once
 
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+#include <cstdio>
+#include <chrono>
 #include <mutex>
 
 #include "qf_common.cuh"
 
 namespace qf {
 
-constexpr int kPagesPerStage = 8;                 // one page per consumer warp
-constexpr int kConsumerWarps = kPagesPerStage;
+#ifndef QF_PAGES_PER_STAGE
+#define QF_PAGES_PER_STAGE 8
+#endif
+#ifndef QF_STAGES
+#define QF_STAGES (24 / QF_PAGES_PER_STAGE)
+#endif
+constexpr int kConsumerWarps = 8;
+constexpr int kPagesPerStage = QF_PAGES_PER_STAGE;          // pages (of one KV head) per ring stage: 8, 4 or 2
+constexpr int kTeams         = kConsumerWarps / kPagesPerStage;  // warp teams that take stages in turn
+constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kSweepThreads  = (kConsumerWarps + 1) * 32;
-constexpr int kStages        = 3;
+constexpr int kStages        = QF_STAGES;
+static_assert(kPagesPerStage == 8 || kPagesPerStage == 4 || kPagesPerStage == 2, "stage must hold 8, 4 or 2 pages");
 constexpr int kMaxSweepCtas  = 512;               // bound used for scratch sizing
 constexpr int kHalfTileBytes = 2048;              // 16 rows x 64 channels of bf16
-constexpr int kStageKVBytes  = kPagesPerStage * kPageBytes * 2;  // K and V
 constexpr int kRedStride     = kHeadDim + 4;      // padded row of the warp-merge buffer
+constexpr int kMaxSmemEntries = 2048;             // (request, shard) pairs planned in shared memory
 constexpr unsigned kSpinLimit = 1u << 24;
 
 struct WorkspaceLayout {
-    size_t header_off, prefix_off, seg_off, total;
+    size_t header_off, prefix_off, counter_off, seg_off, total;
     int seg_stride;  // floats per segment slot
 };
-
-// Header words (int32) at the start of the workspace.
-enum { kHdrStatus = 0, kHdrTotalUnits = 1, kHdrUnitsPerCta = 2 };
 
 inline int seg_stride_floats(int G) { return G * kHeadDim + ((2 * G + 3) & ~3); }
 
@@ -57,7 +69,8 @@ inline WorkspaceLayout workspace_layout(int batch, int max_shards, int num_kv_he
     const size_t entries = (size_t)batch * max_shards;
     L.header_off = 0;
     L.prefix_off = 256;
-    L.seg_off = up(L.prefix_off + (entries + 1) * sizeof(int));
+    L.counter_off = up(L.prefix_off + (entries + 1) * sizeof(int));
+    L.seg_off = up(L.counter_off + entries * num_kv_heads * sizeof(unsigned long long));
     L.seg_stride = seg_stride_floats(G);
     const size_t slots = entries * num_kv_heads + kMaxSweepCtas;
     L.total = up(L.seg_off + slots * L.seg_stride * sizeof(float));
@@ -103,11 +116,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     return false;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+// One (page, KV head) block: 64 channels x 16 rows x 2 halves = 4 KB in one request.
+__device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap *map, int row, uint32_t bar)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(0), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
 {
@@ -151,28 +165,29 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
-// ------------------------------------------------------------------ plan kernel
-// prefix[e] = number of stage units (x Hkv) before entry e = b*S + s.
+// Stage units of entry e = (request, shard), all KV heads together.
+__device__ __forceinline__ int entry_units(const int *__restrict__ seq_lens, const int *__restrict__ shard_ranges,
+                                           int e, int max_shards, int num_kv_heads)
+{
+    int beg, end;
+    clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[e / max_shards], beg, end);
+    if (end <= beg) return 0;
+    const int npages = ((end - 1) >> 4) - (beg >> 4) + 1;
+    return ((npages + kPagesPerStage - 1) / kPagesPerStage) * num_kv_heads;
+}
+
+// ------------------------------------------------------------------ plan kernel (large batches only)
+// prefix[e] = number of stage units before entry e = b*S + s, left in scratch.
 __global__ void __launch_bounds__(1024)
-plan_kernel(const int *__restrict__ seq_lens, const int *__restrict__ shard_ranges, int *__restrict__ header,
-            int *__restrict__ prefix, int n_entries, int max_shards, int num_kv_heads, int n_ctas)
+plan_kernel(const int *__restrict__ seq_lens, const int *__restrict__ shard_ranges, int *__restrict__ prefix,
+            int n_entries, int max_shards, int num_kv_heads)
 {
     __shared__ int warp_sums[32];
-    __shared__ int carry_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) carry_s = 0;
-    __syncthreads();
+    int carry = 0;
     for (int base = 0; base < n_entries; base += 1024) {
         const int e = base + tid;
-        int cnt = 0;
-        if (e < n_entries) {
-            int beg, end;
-            clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[e / max_shards], beg, end);
-            if (end > beg) {
-                const int npages = ((end - 1) >> 4) - (beg >> 4) + 1;
-                cnt = ((npages + kPagesPerStage - 1) / kPagesPerStage) * num_kv_heads;
-            }
-        }
+        const int cnt = (e < n_entries) ? entry_units(seq_lens, shard_ranges, e, max_shards, num_kv_heads) : 0;
         int x = cnt;  // inclusive scan within the warp
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -181,30 +196,17 @@ plan_kernel(const int *__restrict__ seq_lens, const int *__restrict__ shard_rang
         }
         if (lane == 31) warp_sums[warp] = x;
         __syncthreads();
-        if (warp == 0) {
-            int w = warp_sums[lane];
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int y = __shfl_up_sync(0xffffffffu, w, off);
-                if (lane >= off) w += y;
-            }
-            warp_sums[lane] = w;  // inclusive over warps
+        int before = 0, chunk = 0;
+        for (int w = 0; w < 32; ++w) {
+            const int v = warp_sums[w];
+            if (w < warp) before += v;
+            chunk += v;
         }
-        __syncthreads();
-        const int carry = carry_s;
-        const int excl = carry + (warp ? warp_sums[warp - 1] : 0) + x - cnt;
-        if (e < n_entries) prefix[e] = excl;
-        __syncthreads();
-        if (tid == 1023) carry_s = carry + warp_sums[31];
+        if (e < n_entries) prefix[e] = carry + before + x - cnt;
+        carry += chunk;
         __syncthreads();
     }
-    if (tid == 0) {
-        const int total = carry_s;
-        prefix[n_entries] = total;
-        header[kHdrStatus] = 0;
-        header[kHdrTotalUnits] = total;
-        header[kHdrUnitsPerCta] = (total + n_ctas - 1) / n_ctas;
-    }
+    if (tid == 0) prefix[n_entries] = carry;
 }
 
 // ------------------------------------------------------------------ sweep kernel
@@ -215,16 +217,16 @@ struct __align__(16) StageMeta {
     int npages;    // 1..8
     int tok_beg;   // clamped shard range
     int tok_end;
-    int flags;     // bit0 first stage of a segment, bit1 last stage, bit2 segment == whole unit
-    int aux;       // bits 0..7: pages whose table entry was out of range; bits 8..: segment slot
+    int flags;     // bit0 first stage of a segment, bit1 last stage; bits 8..: segments the unit is cut into
+    int aux;       // bits 0..7: pages whose table entry was out of range; bits 8..: first segment slot of the unit
 };
-enum { kSegFirst = 1, kSegLast = 2, kSegWhole = 4 };
+enum { kSegFirst = 1, kSegLast = 2 };
 
 template <int G>
 struct SweepSmem {
     // every K/V half tile is a 1024-byte-aligned 128B-swizzled TMA destination
     alignas(1024) uint8_t kv[kStages][2][kPagesPerStage][kPageBytes];  // [stage][K|V][page][half][row][128B]
-    alignas(16) uint16_t q[kStages][8 * kHeadDim];
+    alignas(16) uint16_t q[kStages][G * kHeadDim];
     static constexpr int kRoundHeads = G < 4 ? G : 4;  // heads merged per epilogue round
     alignas(16) float red_acc[kConsumerWarps][kRoundHeads][kRedStride];
     alignas(16) float red_ml[kConsumerWarps][G][2];
@@ -233,7 +235,40 @@ struct SweepSmem {
     alignas(8) unsigned long long empty_bar[kStages];
     alignas(8) unsigned long long red_bar[2];
     int abort_flag;
+    int is_last;
+    int scan_ws[kConsumerWarps + 1];
+    int prefix[kMaxSmemEntries + 1];
 };
+
+// Merge segments [first, first+nseg) of one (shard, KV head) unit into its final state.
+// Called by all consumer threads of the CTA that arrived last; fixed order, so deterministic.
+template <int G>
+__device__ __forceinline__ void merge_segments(const float *__restrict__ seg, int seg_stride, int first_slot,
+                                               int nseg, size_t out_row, float *__restrict__ o_part,
+                                               float *__restrict__ m_part, float *__restrict__ lse_part, int tid)
+{
+    const float kLn2 = 0.6931471805599453f;
+    for (int idx = tid; idx < G * kHeadDim; idx += kConsumerThreads) {
+        const int head = idx >> 7, d = idx & 127;
+        float M = neg_inf();
+        for (int i = 0; i < nseg; ++i)
+            M = fmaxf(M, __ldcg(seg + (size_t)(first_slot + i) * seg_stride + G * kHeadDim + 2 * head));
+        const bool empty = (M == neg_inf());
+        const float Ms = empty ? 0.f : M;
+        float z = 0.f, wsum = 0.f;
+        for (int i = 0; i < nseg; ++i) {
+            const float *sl = seg + (size_t)(first_slot + i) * seg_stride;
+            const float ew = fast_exp2(__ldcg(sl + G * kHeadDim + 2 * head) - Ms);
+            z = fmaf(__ldcg(sl + G * kHeadDim + 2 * head + 1), ew, z);
+            wsum = fmaf(__ldcg(sl + head * kHeadDim + d), ew, wsum);
+        }
+        o_part[(out_row + head) * kHeadDim + d] = empty ? 0.f : wsum / z;
+        if (d == 0) {
+            m_part[out_row + head] = empty ? neg_inf() : M * kLn2;
+            lse_part[out_row + head] = empty ? neg_inf() : (M + log2f(z)) * kLn2;
+        }
+    }
+}
 
 template <int G>
 __global__ void __launch_bounds__(kSweepThreads, 1)
@@ -241,8 +276,9 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
              const uint16_t *__restrict__ q, const int *__restrict__ block_table,
              const int *__restrict__ seq_lens, const int *__restrict__ shard_ranges,
              float *__restrict__ o_part, float *__restrict__ m_part, float *__restrict__ lse_part,
-             int *__restrict__ header, const int *__restrict__ prefix, float *__restrict__ seg,
-             int seg_stride, DevParams P)
+             unsigned long long *__restrict__ header, const int *__restrict__ global_prefix,
+             unsigned long long *__restrict__ counters, float *__restrict__ seg, int seg_stride,
+             unsigned long long epoch, DevParams P)
 {
     extern __shared__ uint8_t smem_raw[];
     SweepSmem<G> &sm = *reinterpret_cast<SweepSmem<G> *>(
@@ -250,6 +286,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = P.max_shards, Hkv = P.num_kv_heads, Hq = P.num_q_heads;
+    const int n_entries = P.batch * S;
     volatile int *abort_flag = &sm.abort_flag;
 
     if (tid == 0) {
@@ -260,15 +297,52 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
         mbar_init(smem_u32(&sm.red_bar[0]), kConsumerWarps);
         mbar_init(smem_u32(&sm.red_bar[1]), kConsumerWarps);
         sm.abort_flag = 0;
+        sm.is_last = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (blockIdx.x == 0) header[kHdrLastEpoch] = epoch;
     }
-    __syncthreads();
 
-    const int total = header[kHdrTotalUnits];
-    const int per_cta = header[kHdrUnitsPerCta];
+    // ---- plan: prefix sum over (request, shard) entries, in shared memory when it fits
+    const int *prefix;
+    if (global_prefix) {
+        prefix = global_prefix;
+        __syncthreads();
+    } else {
+        int carry = 0;
+        for (int base = 0; base < n_entries; base += kConsumerThreads) {
+            const int e = base + tid;
+            const int cnt = (tid < kConsumerThreads && e < n_entries)
+                                ? entry_units(seq_lens, shard_ranges, e, S, Hkv) : 0;
+            int x = cnt;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, x, off);
+                if (lane >= off) x += y;
+            }
+            if (lane == 31) sm.scan_ws[warp] = x;
+            __syncthreads();
+            int before = 0, chunk = 0;
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w) {
+                const int v = sm.scan_ws[w];
+                if (w < warp) before += v;
+                chunk += v;
+            }
+            if (tid < kConsumerThreads && e < n_entries) sm.prefix[e] = carry + before + x - cnt;
+            carry += chunk;
+            __syncthreads();
+        }
+        if (tid == 0) sm.prefix[n_entries] = carry;
+        __syncthreads();
+        prefix = sm.prefix;
+    }
+    const int total = prefix[n_entries];
+    const int per_cta = (total + (int)gridDim.x - 1) / (int)gridDim.x;
     const long long pos0_ll = (long long)blockIdx.x * per_cta;
     const int pos0 = (int)min((long long)total, pos0_ll);
     const int pos1 = (int)min((long long)total, pos0_ll + per_cta);
+    if (blockIdx.x == 0 && tid == 0)
+        header[kHdrTotals] = (unsigned long long)(unsigned)total | ((unsigned long long)(unsigned)per_cta << 32);
 
     if (warp == kConsumerWarps) {
         // ============================ producer warp ============================
@@ -276,7 +350,6 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
         uint32_t phase = 0;
         int issued = 0;
         bool ok = true;
-        const int n_entries = P.batch * S;
         int pos = pos0;
         int e = 0;
         if (pos < pos1) {  // largest e with prefix[e] <= pos
@@ -298,26 +371,30 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             int beg, end;
             clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[b], beg, end);
             const int first_page = beg >> 4, last_page = (end - 1) >> 4;
-            const bool whole = (j == 0 && seg_len == nunits);
-            const int slot = e * Hkv + c + (int)blockIdx.x;
+            // the CTAs whose slices touch this unit: one segment each
+            const int p0 = base + c * nunits;
+            const int first_cta = p0 / per_cta, last_cta = (p0 + nunits - 1) / per_cta;
+            const int nseg = last_cta - first_cta + 1;
+            const int first_slot = e * Hkv + c + first_cta;
             const long long row_base = (long long)b * P.max_pages_per_req;
 
-            // table entries are fetched 32 pages (4 stages) at a time
+            // table entries are fetched 32 pages at a time
             int tbl_page0 = 0, tbl = 0;
             for (int u = 0; ok && u < seg_len; ++u) {
                 const int page0 = first_page + (j + u) * kPagesPerStage;
                 const int np = min(kPagesPerStage, last_page + 1 - page0);
-                if ((u & 3) == 0) {
+                if ((u & (32 / kPagesPerStage - 1)) == 0) {
                     tbl_page0 = page0;
                     const int lp = min(page0 + lane, last_page);
                     tbl = block_table ? block_table[row_base + lp] : (int)(row_base + lp);
                 }
-                const int i = lane & 7;           // page within the stage
-                const int part = lane >> 3;       // 0: K lo, 1: K hi, 2: V lo, 3: V hi
+                const int i = lane % kPagesPerStage;    // page within the stage
+                const int part = lane / kPagesPerStage; // 0: K page, 1: V page (>= 2: idle lane)
                 int phys = __shfl_sync(0xffffffffu, tbl, (page0 - tbl_page0) + i);
                 bool bad = false;
                 if (P.check_bounds && (phys < 0 || (long long)phys >= P.num_pages)) { bad = true; phys = 0; }
                 const unsigned bad_mask = __ballot_sync(0xffffffffu, bad && i < np && part == 0) & 0xffu;
+                const bool issuer = (i < np) && (part < 2);
 
                 if (!mbar_wait(smem_u32(&sm.empty_bar[stage]), phase ^ 1, abort_flag)) { ok = false; break; }
                 const bool first = (u == 0), last = (u == seg_len - 1);
@@ -326,17 +403,16 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                     StageMeta mt;
                     mt.entry = e; mt.kv_head = c; mt.page0 = page0; mt.npages = np;
                     mt.tok_beg = beg; mt.tok_end = end;
-                    mt.flags = (first ? kSegFirst : 0) | (last ? kSegLast : 0) | (whole ? kSegWhole : 0);
-                    mt.aux = (int)bad_mask | (slot << 8);
+                    mt.flags = (first ? kSegFirst : 0) | (last ? kSegLast : 0) | (nseg << 8);
+                    mt.aux = (int)bad_mask | (first_slot << 8);
                     sm.meta[stage] = mt;
                     mbar_arrive_expect_tx(full, (uint32_t)np * 2u * kPageBytes + (first ? (uint32_t)G * 256u : 0u));
-                    if (bad_mask) atomicOr(header + kHdrStatus, kStatusBadPage);
+                    if (bad_mask) epoch_or(header + kHdrStatus, epoch, kStatusBadPage);
                 }
                 __syncwarp();
-                if (i < np) {
+                if (issuer) {
                     const int row = (phys * Hkv + c) * kPageSize;
-                    const uint32_t dst = smem_u32(&sm.kv[stage][part >> 1][i][0]) + (part & 1) * kHalfTileBytes;
-                    tma_load_2d(dst, (part >> 1) ? &v_map : &k_map, (part & 1) * 64, row, full);
+                    tma_load_page(smem_u32(&sm.kv[stage][part][i][0]), part ? &v_map : &k_map, row, full);
                 }
                 if (first && lane == 0)
                     bulk_load_1d(smem_u32(&sm.q[stage][0]), q + ((size_t)b * Hq + (size_t)c * G) * kHeadDim,
@@ -358,7 +434,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
         }
         if (!ok) {
             // give up: flag it, then wait (bounded) for the copies still in flight
-            if (lane == 0) { sm.abort_flag = 1; atomicOr(header + kHdrStatus, kStatusTimeout); }
+            if (lane == 0) { sm.abort_flag = 1; epoch_or(header + kHdrStatus, epoch, kStatusTimeout); }
             __syncwarp();
             int s2 = stage;
             uint32_t ph2 = phase;
@@ -372,6 +448,17 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     }
 
     // ================================ consumer warps ================================
+    // empty shards: (0, -inf, -inf), spread over all CTAs' consumer warps while the ring fills
+    for (int e = (int)blockIdx.x * kConsumerWarps + warp; e < n_entries; e += (int)gridDim.x * kConsumerWarps) {
+        if (prefix[e + 1] != prefix[e]) continue;
+        float4 *o4 = reinterpret_cast<float4 *>(o_part + (size_t)e * Hq * kHeadDim);
+        for (int i = lane; i < Hq * (kHeadDim / 4); i += 32) o4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int h = lane; h < Hq; h += 32) {
+            m_part[(size_t)e * Hq + h] = neg_inf();
+            lse_part[(size_t)e * Hq + h] = neg_inf();
+        }
+    }
+
     const int g = lane >> 2, t = lane & 3;
     const float scale2 = P.sm_scale * 1.4426950408889634f;  // scores are kept in units of log 2
     const float kLn2 = 0.6931471805599453f;
@@ -379,12 +466,25 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     float m2[2] = {neg_inf(), neg_inf()};
     float l[2] = {0.f, 0.f};
     float acc[8][4];
-    int stage = 0;
-    uint32_t phase = 0, red_phase = 0;
+    int stage = 0, seq = 0;
+    uint32_t phase = 0, red_phase0 = 0, red_phase1 = 0;
+    const int team = warp / kPagesPerStage, wp = warp % kPagesPerStage;  // teams take stages in turn
+
+    // every consumer warp waits on the warp-merge barriers through this; false = abort
+    auto red_sync = [&](int which, uint32_t &ph) -> bool {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sm.red_bar[which]));
+        if (!mbar_wait(smem_u32(&sm.red_bar[which]), ph, abort_flag)) {
+            if (lane == 0) { sm.abort_flag = 1; epoch_or(header + kHdrStatus, epoch, kStatusTimeout); }
+            return false;
+        }
+        ph ^= 1;
+        return true;
+    };
 
     for (;;) {
         if (!mbar_wait(smem_u32(&sm.full_bar[stage]), phase, abort_flag)) {
-            if (lane == 0) { sm.abort_flag = 1; atomicOr(header + kHdrStatus, kStatusTimeout); }
+            if (lane == 0) { sm.abort_flag = 1; epoch_or(header + kHdrStatus, epoch, kStatusTimeout); }
             return;
         }
         const StageMeta mt = sm.meta[stage];
@@ -403,18 +503,24 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             for (int i = 0; i < 8; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
         }
 
-        if (warp < mt.npages) {
-            const int tok0 = (mt.page0 + warp) << 4;
+        const bool my_turn = (kTeams == 1) || ((seq % kTeams) == team);
+        ++seq;
+#ifdef QF_EXP_NOCOMPUTE
+        if (false) {
+#else
+        if (my_turn && wp < mt.npages) {
+#endif
+            const int tok0 = (mt.page0 + wp) << 4;
             int tlo = max(mt.tok_beg - tok0, 0), thi = min(mt.tok_end - tok0, kPageSize);
-            if ((mt.aux >> warp) & 1) { tlo = 0; thi = 0; }
+            if ((mt.aux >> wp) & 1) { tlo = 0; thi = 0; }
             const bool ragged = (tlo > 0) || (thi < kPageSize);
-            const uint32_t k_base = smem_u32(&sm.kv[stage][0][warp][0]);
-            const uint32_t v_base = smem_u32(&sm.kv[stage][1][warp][0]);
+            const uint32_t k_base = smem_u32(&sm.kv[stage][0][wp][0]);
+            const uint32_t v_base = smem_u32(&sm.kv[stage][1][wp][0]);
 
             if (ragged) {
                 // tokens outside the range must contribute nothing, whatever bits they hold:
                 // their value rows are cleared (0 * NaN would poison the product)
-                uint8_t *vb = &sm.kv[stage][1][warp][0];
+                uint8_t *vb = &sm.kv[stage][1][wp][0];
                 for (int idx = lane; idx < kPageBytes / 16; idx += 32) {
                     const int row = (idx >> 3) & 15;
                     if (row < tlo || row >= thi) reinterpret_cast<uint4 *>(vb)[idx] = make_uint4(0, 0, 0, 0);
@@ -425,6 +531,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             // ---- S[token, head] = K Q^T: A = K tile (row major), B = Q^T fragments
             float sc[4] = {0.f, 0.f, 0.f, 0.f};
             {
+                float sc_odd[4] = {0.f, 0.f, 0.f, 0.f};  // two accumulators: half the dependent-MMA chain
                 const int row = (lane & 7) + ((lane >> 3) & 1) * 8;
                 const int csel = lane >> 4;
 #pragma unroll
@@ -434,8 +541,11 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                                           (((chunk & 7) ^ (row & 7)) << 4);
                     uint32_t a[4];
                     ldmatrix_x4(a, addr);
-                    mma_bf16(sc, a, qf[ks][0], qf[ks][1]);
+                    if (ks & 1) mma_bf16(sc_odd, a, qf[ks][0], qf[ks][1]);
+                    else mma_bf16(sc, a, qf[ks][0], qf[ks][1]);
                 }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sc[i] += sc_odd[i];
             }
             // sc[0],sc[1]: token g, heads 2t,2t+1;  sc[2],sc[3]: token g+8
 #pragma unroll
@@ -500,8 +610,12 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                 l[1] += __shfl_xor_sync(0xffffffffu, l[1], off);
             }
             constexpr int RG = SweepSmem<G>::kRoundHeads;
+            const int nseg = mt.flags >> 8;
+            const int first_slot = mt.aux >> 8;
+            const int unit = mt.entry * Hkv + mt.kv_head;
             const size_t out_row = ((size_t)mt.entry * Hq + (size_t)mt.kv_head * G);  // + head
-            float *seg_slot = seg + (size_t)(mt.aux >> 8) * seg_stride;
+            // this CTA's segment is the (blockIdx.x - first_cta)-th of the unit; first_slot = unit + first_cta
+            float *seg_slot = seg + (size_t)(unit + (int)blockIdx.x) * seg_stride;
 #pragma unroll
             for (int hr = 0; hr < G / RG; ++hr) {
 #pragma unroll
@@ -516,13 +630,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                         if (g == 0) { sm.red_ml[warp][head][0] = m2[hh]; sm.red_ml[warp][head][1] = l[hh]; }
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sm.red_bar[0]));
-                if (!mbar_wait(smem_u32(&sm.red_bar[0]), red_phase, abort_flag)) {
-                    if (lane == 0) { sm.abort_flag = 1; atomicOr(header + kHdrStatus, kStatusTimeout); }
-                    return;
-                }
-                for (int idx = tid; idx < RG * kHeadDim; idx += kConsumerWarps * 32) {
+                if (!red_sync(0, red_phase0)) return;
+                for (int idx = tid; idx < RG * kHeadDim; idx += kConsumerThreads) {
                     const int hl = idx >> 7, d = idx & 127;
                     const int head = hr * RG + hl;
                     float M = neg_inf();
@@ -536,7 +645,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                         z = fmaf(sm.red_ml[w][head][1], ew, z);
                         wsum = fmaf(sm.red_acc[w][hl][d], ew, wsum);
                     }
-                    if (mt.flags & kSegWhole) {
+                    if (nseg == 1) {
                         const bool empty = (M == neg_inf());
                         o_part[(out_row + head) * kHeadDim + d] = empty ? 0.f : wsum / z;
                         if (d == 0) {
@@ -544,76 +653,33 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                             lse_part[out_row + head] = empty ? neg_inf() : (M + log2f(z)) * kLn2;
                         }
                     } else {
-                        seg_slot[head * kHeadDim + d] = wsum;
+                        __stcg(seg_slot + head * kHeadDim + d, wsum);
                         if (d == 0) {
-                            seg_slot[G * kHeadDim + 2 * head] = M;
-                            seg_slot[G * kHeadDim + 2 * head + 1] = z;
+                            __stcg(seg_slot + G * kHeadDim + 2 * head, M);
+                            __stcg(seg_slot + G * kHeadDim + 2 * head + 1, z);
                         }
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sm.red_bar[1]));
-                if (!mbar_wait(smem_u32(&sm.red_bar[1]), red_phase, abort_flag)) {
-                    if (lane == 0) { sm.abort_flag = 1; atomicOr(header + kHdrStatus, kStatusTimeout); }
-                    return;
+                if (nseg > 1) __threadfence();   // segment state visible device-wide before the arrival below
+                if (!red_sync(1, red_phase1)) return;
+            }
+            if (nseg > 1) {
+                // the unit was cut by slice boundaries: whoever arrives last merges all its segments
+                if (tid == 0) {
+                    const unsigned n = epoch_arrive(counters + unit, epoch);
+                    if (n == 0) epoch_or(header + kHdrStatus, epoch, kStatusTimeout);
+                    sm.is_last = (n == (unsigned)nseg) ? 1 : 0;
                 }
-                red_phase ^= 1;
+                if (!red_sync(0, red_phase0)) return;
+                const int is_last = *reinterpret_cast<volatile int *>(&sm.is_last);
+                if (is_last) {
+                    __threadfence();
+                    merge_segments<G>(seg, seg_stride, first_slot, nseg, out_row, o_part, m_part, lse_part, tid);
+                }
+                if (!red_sync(1, red_phase1)) return;
             }
         }
         if (++stage == kStages) { stage = 0; phase ^= 1; }
-    }
-}
-
-// ------------------------------------------------------------------ merge kernel
-// One CTA per (request, shard, KV head); thread = channel.  Merges the segment
-// states a (shard, KV head) was split into by CTA-slice boundaries, and writes
-// the empty-shard convention (o = 0, m = lse = -inf).
-template <int G>
-__global__ void __launch_bounds__(kHeadDim)
-merge_kernel(const int *__restrict__ header, const int *__restrict__ prefix, const float *__restrict__ seg,
-             int seg_stride, float *__restrict__ o_part, float *__restrict__ m_part,
-             float *__restrict__ lse_part, int num_q_heads, int num_kv_heads)
-{
-    const int c = blockIdx.x;
-    const int e = blockIdx.y;
-    const int d = threadIdx.x;
-    const float kLn2 = 0.6931471805599453f;
-    const int base = prefix[e];
-    const int cnt = prefix[e + 1] - base;
-    const size_t out_row = (size_t)e * num_q_heads + (size_t)c * G;
-    if (cnt == 0) {
-#pragma unroll
-        for (int h = 0; h < G; ++h) {
-            o_part[(out_row + h) * kHeadDim + d] = 0.f;
-            if (d == 0) { m_part[out_row + h] = neg_inf(); lse_part[out_row + h] = neg_inf(); }
-        }
-        return;
-    }
-    const int nunits = cnt / num_kv_heads;
-    const int per_cta = header[kHdrUnitsPerCta];
-    const int p0 = base + c * nunits, p1 = p0 + nunits;
-    const int first = p0 / per_cta, last = (p1 - 1) / per_cta;
-    if (first == last) return;  // the sweep wrote this state directly
-    const int unit = e * num_kv_heads + c;
-#pragma unroll
-    for (int h = 0; h < G; ++h) {
-        float M = neg_inf();
-        for (int i = first; i <= last; ++i)
-            M = fmaxf(M, seg[(size_t)(unit + i) * seg_stride + G * kHeadDim + 2 * h]);
-        const bool empty = (M == neg_inf());
-        const float Ms = empty ? 0.f : M;
-        float z = 0.f, wsum = 0.f;
-        for (int i = first; i <= last; ++i) {
-            const float *sl = seg + (size_t)(unit + i) * seg_stride;
-            const float ew = fast_exp2(sl[G * kHeadDim + 2 * h] - Ms);
-            z = fmaf(sl[G * kHeadDim + 2 * h + 1], ew, z);
-            wsum = fmaf(sl[h * kHeadDim + d], ew, wsum);
-        }
-        o_part[(out_row + h) * kHeadDim + d] = empty ? 0.f : wsum / z;
-        if (d == 0) {
-            m_part[out_row + h] = empty ? neg_inf() : M * kLn2;
-            lse_part[out_row + h] = empty ? neg_inf() : (M + log2f(z)) * kLn2;
-        }
     }
 }
 
@@ -623,7 +689,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 
-// A [rows, 128] bf16 view of a KV pool, boxes of 16 rows x 64 channels, 128B swizzle.
+// A [2 halves, rows, 64] bf16 view of a KV pool, one 4 KB box per (page, KV head), 128B swizzle.
 inline int make_pool_map(CUtensorMap *out, const void *pool, long long num_pages, int num_kv_heads, char *msg,
                          size_t msg_len)
 {
@@ -648,12 +714,14 @@ inline int make_pool_map(CUtensorMap *out, const void *pool, long long num_pages
         }
         encode = (EncodeTiledFn)fn;
     }
-    const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)num_pages * num_kv_heads * kPageSize};
-    const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kPageSize};
-    const cuuint32_t estr[2] = {1, 1};
+    // dims: 64 channels (128 B, the swizzle span), rows (256 B apart), the two halves of a row (128 B apart);
+    // a box is one whole 4 KB (page, KV head) block, landing in shared memory as [half][row][128 B]
+    const cuuint64_t dims[3] = {64, (cuuint64_t)num_pages * num_kv_heads * kPageSize, 2};
+    const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kPageSize, 2};
+    const cuuint32_t estr[3] = {1, 1, 1};
     CUtensorMap map;
-    CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box,
+    CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(pool), dims, strides, box,
                         estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -668,14 +736,23 @@ inline int make_pool_map(CUtensorMap *out, const void *pool, long long num_pages
     return 0;
 }
 
+// A fresh 54-bit tag per launch: process-random high part, counter low part.
+inline unsigned long long next_epoch()
+{
+    static std::atomic<unsigned long long> counter{
+        ((unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count() * 0x9E3779B97F4A7C15ull) >> 10};
+    return (counter.fetch_add(1) + 1) & ((1ull << 54) - 1);
+}
+
 template <int G>
 int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void *q, const int32_t *bt,
                    const int32_t *sl, const int32_t *sr, float *o, float *m, float *l, const DevParams &P,
-                   char *ws, const WorkspaceLayout &wsl, int n_ctas, cudaStream_t st, cudaEvent_t ev0,
-                   cudaEvent_t ev1, char *msg, size_t msg_len, int *launches)
+                   char *ws, const WorkspaceLayout &wsl, int n_ctas, unsigned long long epoch, cudaStream_t st,
+                   cudaEvent_t ev0, cudaEvent_t ev1, char *msg, size_t msg_len, int *launches)
 {
-    int *header = reinterpret_cast<int *>(ws + wsl.header_off);
+    unsigned long long *header = reinterpret_cast<unsigned long long *>(ws + wsl.header_off);
     int *prefix = reinterpret_cast<int *>(ws + wsl.prefix_off);
+    unsigned long long *counters = reinterpret_cast<unsigned long long *>(ws + wsl.counter_off);
     float *seg = reinterpret_cast<float *>(ws + wsl.seg_off);
     const int n_entries = P.batch * P.max_shards;
     const size_t smem = sizeof(SweepSmem<G>) + 1024;
@@ -687,38 +764,40 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
         if (e != cudaSuccess) { snprintf(msg, msg_len, "cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return -5; }
         attr_set[dev & 63] = true;
     }
-    plan_kernel<<<1, 1024, 0, st>>>(sl, sr, header, prefix, n_entries, P.max_shards, P.num_kv_heads, n_ctas);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) { snprintf(msg, msg_len, "plan_kernel launch: %s", cudaGetErrorString(e)); return -5; }
+    *launches = 0;
+    const int *global_prefix = nullptr;
+    if (n_entries > kMaxSmemEntries) {
+        plan_kernel<<<1, 1024, 0, st>>>(sl, sr, prefix, n_entries, P.max_shards, P.num_kv_heads);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) { snprintf(msg, msg_len, "plan_kernel launch: %s", cudaGetErrorString(e)); return -5; }
+        global_prefix = prefix;
+        *launches += 1;
+    }
     if (ev0) cudaEventRecord(ev0, st);
     sweep_kernel<G><<<n_ctas, kSweepThreads, smem, st>>>(kmap, vmap, (const uint16_t *)q, bt, sl, sr, o, m, l,
-                                                          header, prefix, seg, wsl.seg_stride, P);
-    e = cudaGetLastError();
+                                                          header, global_prefix, counters, seg, wsl.seg_stride,
+                                                          epoch, P);
+    cudaError_t e = cudaGetLastError();
     if (ev1) cudaEventRecord(ev1, st);
     if (e != cudaSuccess) { snprintf(msg, msg_len, "sweep_kernel launch: %s", cudaGetErrorString(e)); return -5; }
-    dim3 mgrid(P.num_kv_heads, n_entries);
-    merge_kernel<G><<<mgrid, kHeadDim, 0, st>>>(header, prefix, seg, wsl.seg_stride, o, m, l, P.num_q_heads,
-                                                P.num_kv_heads);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) { snprintf(msg, msg_len, "merge_kernel launch: %s", cudaGetErrorString(e)); return -5; }
-    *launches = 3;
+    *launches += 1;
     return 0;
 }
 
 inline int launch_sweep(const void *q, const void *k_cache, const void *v_cache, const int32_t *bt,
                         const int32_t *sl, const int32_t *sr, float *o, float *m, float *l, const DevParams &P,
-                        char *ws, const WorkspaceLayout &wsl, int sm_count, cudaStream_t st, cudaEvent_t ev0,
-                        cudaEvent_t ev1, char *msg, size_t msg_len, int *launches)
+                        char *ws, const WorkspaceLayout &wsl, int sm_count, unsigned long long epoch,
+                        cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1, char *msg, size_t msg_len, int *launches)
 {
     CUtensorMap kmap, vmap;
     if (make_pool_map(&kmap, k_cache, P.num_pages, P.num_kv_heads, msg, msg_len)) return -5;
     if (make_pool_map(&vmap, v_cache, P.num_pages, P.num_kv_heads, msg, msg_len)) return -5;
     const int n_ctas = sm_count < kMaxSweepCtas ? sm_count : kMaxSweepCtas;
     switch (P.group) {
-    case 1: return launch_sweep_g<1>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, st, ev0, ev1, msg, msg_len, launches);
-    case 2: return launch_sweep_g<2>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, st, ev0, ev1, msg, msg_len, launches);
-    case 4: return launch_sweep_g<4>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, st, ev0, ev1, msg, msg_len, launches);
-    default: return launch_sweep_g<8>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, st, ev0, ev1, msg, msg_len, launches);
+    case 1: return launch_sweep_g<1>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
+    case 2: return launch_sweep_g<2>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
+    case 4: return launch_sweep_g<4>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
+    default: return launch_sweep_g<8>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
     }
 }
 

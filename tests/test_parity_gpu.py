@@ -301,3 +301,16 @@ def test_full_size_configs_sampled(cfg):
     errs = T.compare_sampled(dw, w, seed=cfg, tag=w.name)
     print(w.name, errs)
     assert dw.status() == 0
+
+
+def test_many_entries_plan_in_scratch():
+    # more (request, shard) pairs than the in-kernel plan holds: the separate plan kernel path
+    rng = np.random.default_rng(41)
+    B = 700
+    lens = rng.integers(0, 300, size=B).tolist()
+    ranges = [wl.even_shards(L, 3) + [(0, 0)] for L in lens]   # S = 4 -> 2,800 entries
+    w = wl.make_workload("many", lens, ranges, 4, 2, seed=41, poison_tails=True)
+    assert w.batch * w.max_shards > 2048
+    dw = run(w)
+    T.compare_all(dw, w)
+    assert dw.status() == 0
