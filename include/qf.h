@@ -91,7 +91,11 @@ enum {
 
 enum {
     QF_FLAG_CHECK_BOUNDS  = 1, /* range-check page indices on the device           */
-    QF_FLAG_SIMPLE_KERNEL = 2  /* use the plain-load sweep kernel (validation aid) */
+    QF_FLAG_SIMPLE_KERNEL = 2, /* use the plain-load sweep kernel (validation aid) */
+    QF_FLAG_HEAD_PARALLEL = 4  /* use the head-parallel sweep kernel (needs Hkv a multiple
+                                  of 8 and G <= 4, else ignored): one page of eight KV
+                                  heads per ring stage, no cross-warp merges; faster when
+                                  shards are short (a few hundred tokens to ~2,000)      */
 };
 
 /* qf_read_status bits */

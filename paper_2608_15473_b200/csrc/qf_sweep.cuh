@@ -33,6 +33,7 @@
 #include <mutex>
 
 #include "qf_common.cuh"
+#include "qf_page_math.cuh"
 
 namespace qf {
 
@@ -49,11 +50,10 @@ constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kSweepThreads  = (kConsumerWarps + 1) * 32;
 constexpr int kStages        = QF_STAGES;
 static_assert(kPagesPerStage == 8 || kPagesPerStage == 4 || kPagesPerStage == 2, "stage must hold 8, 4 or 2 pages");
-constexpr int kMaxSweepCtas  = 512;               // bound used for scratch sizing
+constexpr int kMaxSweepCtas  = 160;               // persistent CTAs (one per SM) are capped at this
 constexpr int kHalfTileBytes = 2048;              // 16 rows x 64 channels of bf16
 constexpr int kRedStride     = kHeadDim + 4;      // padded row of the warp-merge buffer
 constexpr int kMaxSmemEntries = 2048;             // (request, shard) pairs planned in shared memory
-constexpr unsigned kSpinLimit = 1u << 24;
 
 struct WorkspaceLayout {
     size_t header_off, prefix_off, counter_off, seg_off, total;
@@ -72,107 +72,25 @@ inline WorkspaceLayout workspace_layout(int batch, int max_shards, int num_kv_he
     L.counter_off = up(L.prefix_off + (entries + 1) * sizeof(int));
     L.seg_off = up(L.counter_off + entries * num_kv_heads * sizeof(unsigned long long));
     L.seg_stride = seg_stride_floats(G);
-    const size_t slots = entries * num_kv_heads + kMaxSweepCtas;
+    // unit kernel: slot = unit + CTA; head-parallel kernel: two slot groups of eight heads per CTA
+    const size_t unit_slots = entries * num_kv_heads + (size_t)kMaxSweepCtas;
+    const size_t hp_slots = (num_kv_heads % 8 == 0 && G <= 4) ? (size_t)kMaxSweepCtas * 2 * 8 : 0;
+    const size_t slots = unit_slots > hp_slots ? unit_slots : hp_slots;
     L.total = up(L.seg_off + slots * L.seg_stride * sizeof(float));
     return L;
 }
 
-// ------------------------------------------------------------------ PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void *p)
-{
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false if the limit ran out or another warp aborted.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
-{
-    for (unsigned it = 0; it < kSpinLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (it > 64) {
-            if (*abort_flag) return false;
-            __nanosleep(64);
-        }
-    }
-    return false;
-}
-// One (page, KV head) block: 64 channels x 16 rows x 2 halves = 4 KB in one request.
-__device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap *map, int row, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(0), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
-{
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr)
-{
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a)
-{
-    uint32_t d;
-    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
-    return d;
-}
-// D = A(16x16, row) * B(16x8, col) + D, bf16 inputs, fp32 accumulate.
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ float fast_exp2(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t *>(&v);
-}
-
-// Stage units of entry e = (request, shard), all KV heads together.
+// Work units of entry e = (request, shard), all KV heads together.  hp_groups == 0: stage units of
+// kPagesPerStage pages per KV head (unit kernel); hp_groups > 0: pages per group of eight KV heads
+// (head-parallel kernel).
 __device__ __forceinline__ int entry_units(const int *__restrict__ seq_lens, const int *__restrict__ shard_ranges,
-                                           int e, int max_shards, int num_kv_heads)
+                                           int e, int max_shards, int num_kv_heads, int hp_groups)
 {
     int beg, end;
     clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[e / max_shards], beg, end);
     if (end <= beg) return 0;
     const int npages = ((end - 1) >> 4) - (beg >> 4) + 1;
+    if (hp_groups > 0) return npages * hp_groups;
     return ((npages + kPagesPerStage - 1) / kPagesPerStage) * num_kv_heads;
 }
 
@@ -180,14 +98,14 @@ __device__ __forceinline__ int entry_units(const int *__restrict__ seq_lens, con
 // prefix[e] = number of stage units before entry e = b*S + s, left in scratch.
 __global__ void __launch_bounds__(1024)
 plan_kernel(const int *__restrict__ seq_lens, const int *__restrict__ shard_ranges, int *__restrict__ prefix,
-            int n_entries, int max_shards, int num_kv_heads)
+            int n_entries, int max_shards, int num_kv_heads, int hp_groups)
 {
     __shared__ int warp_sums[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int carry = 0;
     for (int base = 0; base < n_entries; base += 1024) {
         const int e = base + tid;
-        const int cnt = (e < n_entries) ? entry_units(seq_lens, shard_ranges, e, max_shards, num_kv_heads) : 0;
+        const int cnt = (e < n_entries) ? entry_units(seq_lens, shard_ranges, e, max_shards, num_kv_heads, hp_groups) : 0;
         int x = cnt;  // inclusive scan within the warp
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -241,23 +159,23 @@ struct SweepSmem {
 };
 
 // Merge segments [first, first+nseg) of one (shard, KV head) unit into its final state.
-// Called by all consumer threads of the CTA that arrived last; fixed order, so deterministic.
-template <int G>
+// Called by the NT threads (a warp or all consumer warps) that arrived last; fixed order, so deterministic.
+template <int G, int NT>
 __device__ __forceinline__ void merge_segments(const float *__restrict__ seg, int seg_stride, int first_slot,
-                                               int nseg, size_t out_row, float *__restrict__ o_part,
+                                               int slot_step, int nseg, size_t out_row, float *__restrict__ o_part,
                                                float *__restrict__ m_part, float *__restrict__ lse_part, int tid)
 {
     const float kLn2 = 0.6931471805599453f;
-    for (int idx = tid; idx < G * kHeadDim; idx += kConsumerThreads) {
+    for (int idx = tid; idx < G * kHeadDim; idx += NT) {
         const int head = idx >> 7, d = idx & 127;
         float M = neg_inf();
         for (int i = 0; i < nseg; ++i)
-            M = fmaxf(M, __ldcg(seg + (size_t)(first_slot + i) * seg_stride + G * kHeadDim + 2 * head));
+            M = fmaxf(M, __ldcg(seg + (size_t)(first_slot + i * slot_step) * seg_stride + G * kHeadDim + 2 * head));
         const bool empty = (M == neg_inf());
         const float Ms = empty ? 0.f : M;
         float z = 0.f, wsum = 0.f;
         for (int i = 0; i < nseg; ++i) {
-            const float *sl = seg + (size_t)(first_slot + i) * seg_stride;
+            const float *sl = seg + (size_t)(first_slot + i * slot_step) * seg_stride;
             const float ew = fast_exp2(__ldcg(sl + G * kHeadDim + 2 * head) - Ms);
             z = fmaf(__ldcg(sl + G * kHeadDim + 2 * head + 1), ew, z);
             wsum = fmaf(__ldcg(sl + head * kHeadDim + d), ew, wsum);
@@ -312,7 +230,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
         for (int base = 0; base < n_entries; base += kConsumerThreads) {
             const int e = base + tid;
             const int cnt = (tid < kConsumerThreads && e < n_entries)
-                                ? entry_units(seq_lens, shard_ranges, e, S, Hkv) : 0;
+                                ? entry_units(seq_lens, shard_ranges, e, S, Hkv, 0) : 0;
             int x = cnt;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
@@ -517,86 +435,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             const uint32_t k_base = smem_u32(&sm.kv[stage][0][wp][0]);
             const uint32_t v_base = smem_u32(&sm.kv[stage][1][wp][0]);
 
-            if (ragged) {
-                // tokens outside the range must contribute nothing, whatever bits they hold:
-                // their value rows are cleared (0 * NaN would poison the product)
-                uint8_t *vb = &sm.kv[stage][1][wp][0];
-                for (int idx = lane; idx < kPageBytes / 16; idx += 32) {
-                    const int row = (idx >> 3) & 15;
-                    if (row < tlo || row >= thi) reinterpret_cast<uint4 *>(vb)[idx] = make_uint4(0, 0, 0, 0);
-                }
-                __syncwarp();
-            }
-
-            // ---- S[token, head] = K Q^T: A = K tile (row major), B = Q^T fragments
-            float sc[4] = {0.f, 0.f, 0.f, 0.f};
-            {
-                float sc_odd[4] = {0.f, 0.f, 0.f, 0.f};  // two accumulators: half the dependent-MMA chain
-                const int row = (lane & 7) + ((lane >> 3) & 1) * 8;
-                const int csel = lane >> 4;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const int chunk = 2 * ks + csel;  // 16-byte chunk of the 256-byte row
-                    const uint32_t addr = k_base + (chunk >> 3) * kHalfTileBytes + row * 128 +
-                                          (((chunk & 7) ^ (row & 7)) << 4);
-                    uint32_t a[4];
-                    ldmatrix_x4(a, addr);
-                    if (ks & 1) mma_bf16(sc_odd, a, qf[ks][0], qf[ks][1]);
-                    else mma_bf16(sc, a, qf[ks][0], qf[ks][1]);
-                }
-#pragma unroll
-                for (int i = 0; i < 4; ++i) sc[i] += sc_odd[i];
-            }
-            // sc[0],sc[1]: token g, heads 2t,2t+1;  sc[2],sc[3]: token g+8
-#pragma unroll
-            for (int i = 0; i < 4; ++i) sc[i] *= scale2;
-            if (ragged) {
-                if (g < tlo || g >= thi) { sc[0] = neg_inf(); sc[1] = neg_inf(); }
-                if (g + 8 < tlo || g + 8 >= thi) { sc[2] = neg_inf(); sc[3] = neg_inf(); }
-            }
-            float mx0 = fmaxf(sc[0], sc[2]), mx1 = fmaxf(sc[1], sc[3]);
-#pragma unroll
-            for (int off = 4; off < 32; off <<= 1) {
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
-            }
-            const float mn0 = fmaxf(m2[0], mx0), mn1 = fmaxf(m2[1], mx1);
-            const float ms0 = (mn0 == neg_inf()) ? 0.f : mn0;  // nothing seen yet: avoid inf - inf
-            const float ms1 = (mn1 == neg_inf()) ? 0.f : mn1;
-            const float al0 = fast_exp2(m2[0] - ms0), al1 = fast_exp2(m2[1] - ms1);
-            const float p0 = fast_exp2(sc[0] - ms0), p1 = fast_exp2(sc[1] - ms1);
-            const float p2 = fast_exp2(sc[2] - ms0), p3 = fast_exp2(sc[3] - ms1);
-            m2[0] = mn0; m2[1] = mn1;
-            l[0] = fmaf(l[0], al0, p0 + p2);   // Z from the unrounded weights
-            l[1] = fmaf(l[1], al1, p1 + p3);
-            if (__any_sync(0xffffffffu, (al0 != 1.f) || (al1 != 1.f))) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    acc[i][0] *= al0; acc[i][1] *= al1; acc[i][2] *= al0; acc[i][3] *= al1;
-                }
-            }
-            // P^T as the B operand, split into bf16 hi + lo so that the product keeps ~16 bits
-            const uint32_t h0 = pack_bf16(p0, p1), h1 = pack_bf16(p2, p3);
-            const uint32_t l0 = pack_bf16(p0 - bf16lo_to_f32(h0), p1 - bf16hi_to_f32(h0));
-            const uint32_t l1 = pack_bf16(p2 - bf16lo_to_f32(h1), p3 - bf16hi_to_f32(h1));
-            const uint32_t bh0 = movmatrix_trans(h0), bh1 = movmatrix_trans(h1);
-            const uint32_t bl0 = movmatrix_trans(l0), bl1 = movmatrix_trans(l1);
-
-            // ---- O^T[d, head] += V^T P^T: A = V^T via transposing loads
-            {
-                const int row = (lane & 7) + (lane >> 4) * 8;
-                const int csel = (lane >> 3) & 1;
-#pragma unroll
-                for (int mt_i = 0; mt_i < 8; ++mt_i) {
-                    const int chunk = 2 * mt_i + csel;
-                    const uint32_t addr = v_base + (chunk >> 3) * kHalfTileBytes + row * 128 +
-                                          (((chunk & 7) ^ (row & 7)) << 4);
-                    uint32_t a[4];
-                    ldmatrix_x4_trans(a, addr);
-                    mma_bf16(acc[mt_i], a, bh0, bh1);
-                    mma_bf16(acc[mt_i], a, bl0, bl1);
-                }
-            }
+            process_page(k_base, v_base, kHalfTileBytes, tlo, thi, ragged, qf, m2, l, acc, scale2, lane);
             if (ragged) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         __syncwarp();
@@ -674,7 +513,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                 const int is_last = *reinterpret_cast<volatile int *>(&sm.is_last);
                 if (is_last) {
                     __threadfence();
-                    merge_segments<G>(seg, seg_stride, first_slot, nseg, out_row, o_part, m_part, lse_part, tid);
+                    merge_segments<G, kConsumerThreads>(seg, seg_stride, first_slot, 1, nseg, out_row, o_part, m_part, lse_part, tid);
                 }
                 if (!red_sync(1, red_phase1)) return;
             }
@@ -690,17 +529,19 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapFloatOOBfill);
 
 // A [2 halves, rows, 64] bf16 view of a KV pool, one 4 KB box per (page, KV head), 128B swizzle.
-inline int make_pool_map(CUtensorMap *out, const void *pool, long long num_pages, int num_kv_heads, char *msg,
-                         size_t msg_len)
+// box_rows = 16 boxes one (page, KV head) block (4 KB); 128 boxes eight heads of a page (32 KB).
+inline int make_pool_map(CUtensorMap *out, const void *pool, long long num_pages, int num_kv_heads, int box_rows,
+                         char *msg, size_t msg_len)
 {
     static EncodeTiledFn encode = nullptr;
     static std::mutex mu;
-    struct Entry { const void *pool; long long pages; int heads; CUtensorMap map; };
+    struct Entry { const void *pool; long long pages; int heads; int rows; CUtensorMap map; };
     static Entry cache[16];
     static int n_cached = 0, next = 0;
     std::lock_guard<std::mutex> lock(mu);
     for (int i = 0; i < n_cached; ++i)
-        if (cache[i].pool == pool && cache[i].pages == num_pages && cache[i].heads == num_kv_heads) {
+        if (cache[i].pool == pool && cache[i].pages == num_pages && cache[i].heads == num_kv_heads &&
+            cache[i].rows == box_rows) {
             *out = cache[i].map;
             return 0;
         }
@@ -718,7 +559,7 @@ inline int make_pool_map(CUtensorMap *out, const void *pool, long long num_pages
     // a box is one whole 4 KB (page, KV head) block, landing in shared memory as [half][row][128 B]
     const cuuint64_t dims[3] = {64, (cuuint64_t)num_pages * num_kv_heads * kPageSize, 2};
     const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, 128};
-    const cuuint32_t box[3] = {64, (cuuint32_t)kPageSize, 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 2};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUtensorMap map;
     CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(pool), dims, strides, box,
@@ -729,7 +570,7 @@ inline int make_pool_map(CUtensorMap *out, const void *pool, long long num_pages
         return -1;
     }
     Entry &slot = cache[next];
-    slot.pool = pool; slot.pages = num_pages; slot.heads = num_kv_heads; slot.map = map;
+    slot.pool = pool; slot.pages = num_pages; slot.heads = num_kv_heads; slot.rows = box_rows; slot.map = map;
     next = (next + 1) % 16;
     if (n_cached < 16) ++n_cached;
     *out = map;
@@ -767,7 +608,7 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
     *launches = 0;
     const int *global_prefix = nullptr;
     if (n_entries > kMaxSmemEntries) {
-        plan_kernel<<<1, 1024, 0, st>>>(sl, sr, prefix, n_entries, P.max_shards, P.num_kv_heads);
+        plan_kernel<<<1, 1024, 0, st>>>(sl, sr, prefix, n_entries, P.max_shards, P.num_kv_heads, 0);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) { snprintf(msg, msg_len, "plan_kernel launch: %s", cudaGetErrorString(e)); return -5; }
         global_prefix = prefix;
@@ -790,8 +631,8 @@ inline int launch_sweep(const void *q, const void *k_cache, const void *v_cache,
                         cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1, char *msg, size_t msg_len, int *launches)
 {
     CUtensorMap kmap, vmap;
-    if (make_pool_map(&kmap, k_cache, P.num_pages, P.num_kv_heads, msg, msg_len)) return -5;
-    if (make_pool_map(&vmap, v_cache, P.num_pages, P.num_kv_heads, msg, msg_len)) return -5;
+    if (make_pool_map(&kmap, k_cache, P.num_pages, P.num_kv_heads, kPageSize, msg, msg_len)) return -5;
+    if (make_pool_map(&vmap, v_cache, P.num_pages, P.num_kv_heads, kPageSize, msg, msg_len)) return -5;
     const int n_ctas = sm_count < kMaxSweepCtas ? sm_count : kMaxSweepCtas;
     switch (P.group) {
     case 1: return launch_sweep_g<1>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);

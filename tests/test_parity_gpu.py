@@ -29,15 +29,19 @@ def run(w, flags=0, null_table=False):
     return dw
 
 
-KERNELS = [pytest.param(0, id="staged"), pytest.param(qf.QF_FLAG_SIMPLE_KERNEL, id="simple")]
+# (flags, number of KV heads): the unit kernel is the default; the head-parallel kernel is opt-in and needs
+# KV heads in groups of eight; the plain-load kernel is the validation aid
+KERNELS = [pytest.param((qf.QF_FLAG_HEAD_PARALLEL, 8), id="headpar"), pytest.param((0, 8), id="unit8"),
+           pytest.param((0, 2), id="unit2"), pytest.param((qf.QF_FLAG_SIMPLE_KERNEL, 2), id="simple")]
 
 
 # T1: every short length, both group sizes, shuffled table: tail-page masking, first-tile guard
 @pytest.mark.parametrize("flags", KERNELS)
 @pytest.mark.parametrize("G", [1, 2, 4, 8])
 def test_every_short_length(G, flags):
+    flags, Hkv = flags
     lens = list(range(1, 49))
-    w = wl.make_workload("t1", lens, [[(0, L)] for L in lens], 2 * G, 2, seed=G, poison_tails=True,
+    w = wl.make_workload("t1", lens, [[(0, L)] for L in lens], Hkv * G, Hkv, seed=G, poison_tails=True,
                          pool_factor=1.3, poison_unused=True)
     dw = run(w, flags)
     T.compare_all(dw, w, tag=f"G={G}")
@@ -47,6 +51,7 @@ def test_every_short_length(G, flags):
 # T2: degenerate and unaligned shard ranges, clamping, L = 0, shard_counts < S
 @pytest.mark.parametrize("flags", KERNELS)
 def test_degenerate_shard_ranges(flags):
+    flags, Hkv = flags
     lens = [100, 0, 37, 300, 16, 1]
     ranges = [
         [(0, 7), (7, 7), (7, 33), (33, 100)],
@@ -57,7 +62,7 @@ def test_degenerate_shard_ranges(flags):
         [(0, 1), (1, 1), (0, 0), (0, 0)],
     ]
     counts = [4, 4, 4, 4, 2, 1]
-    w = wl.make_workload("t2", lens, ranges, 8, 2, seed=5, poison_tails=True, shard_counts=counts,
+    w = wl.make_workload("t2", lens, ranges, 4 * Hkv, Hkv, seed=5, poison_tails=True, shard_counts=counts,
                          max_pages_per_req=40)
     dw = run(w, flags)
     T.compare_all(dw, w)
@@ -71,13 +76,14 @@ def test_degenerate_shard_ranges(flags):
 @pytest.mark.parametrize("flags", KERNELS)
 @pytest.mark.parametrize("G", [2, 4])
 def test_planted_dominant_token(G, flags):
+    flags, Hkv = flags
     L = 1500
     shards = [(0, 130), (130, 641), (641, 1024), (1024, 1500)]
     spots = [0, L - 1, 15, 16, 17, 127, 128, 129, 130, 255, 256, 640, 641, 1023, 1024, 1039, 1040, 1279, 1280, 1499 - 16]
     B = len(spots)
-    w = wl.make_workload("t3", [L] * B, [shards] * B, 2 * G, 2, seed=11 + G)
+    w = wl.make_workload("t3", [L] * B, [shards] * B, Hkv * G, Hkv, seed=11 + G)
     for b, pos in enumerate(spots):
-        for c in range(2):
+        for c in range(Hkv):
             w.q[b, c * G:(c + 1) * G] = w.q[b, c * G]      # one query per group, so one key dominates all its heads
             qrow = wl.bf16_bits_to_f32(w.q[b, c * G])
             w.k_cache[w.block_table[b, pos // 16], c, pos % 16] = wl.f32_to_bf16_bits(2.0 * qrow)
@@ -93,9 +99,11 @@ def test_planted_dominant_token(G, flags):
 # T4: NaN poison everywhere the path must not read
 @pytest.mark.parametrize("flags", KERNELS)
 def test_nan_poison_is_never_read(flags):
+    flags, Hkv = flags
     lens = [70, 333, 18]
     ranges = [[(5, 40), (40, 70)], [(3, 200), (200, 321)], [(1, 2), (2, 17)]]
-    w = wl.make_workload("t4", lens, ranges, 8, 2, seed=13, pool_factor=2.0, poison_unused=True, poison_tails=True)
+    w = wl.make_workload("t4", lens, ranges, 4 * Hkv, Hkv, seed=13, pool_factor=2.0, poison_unused=True,
+                         poison_tails=True)
     nan = np.uint16(0x7FC0)
     for b, rr in enumerate(ranges):  # poison the tokens outside every shard range too
         covered = np.zeros(lens[b], bool)
@@ -108,7 +116,7 @@ def test_nan_poison_is_never_read(flags):
     errs = T.compare_all(dw, w)
     assert errs["out"] < T.ENG_OUT
     # empty shards' vectors are never read by the combine
-    w2 = wl.make_workload("t4b", [64], [[(0, 30), (30, 30), (30, 64)]], 4, 2, seed=14)
+    w2 = wl.make_workload("t4b", [64], [[(0, 30), (30, 30), (30, 64)]], 2 * Hkv, Hkv, seed=14)
     dw2 = DeviceWorkload(w2, flags=flags)
     dw2.sweep()
     dw2.o_part[0, 1].fill_(float("nan"))
@@ -150,14 +158,15 @@ def test_paging_invariance_bitwise():
 # T6: extremes: logits near +85, near -85, mixed across shards
 @pytest.mark.parametrize("flags", KERNELS)
 def test_extreme_logits(flags):
+    flags, Hkv = flags
     L = 2048
-    w = wl.make_workload("t6", [L] * 3, [wl.even_shards(L, 4)] * 3, 4, 2, seed=19, table="shuffled")
+    w = wl.make_workload("t6", [L] * 3, [wl.even_shards(L, 4)] * 3, 2 * Hkv, Hkv, seed=19, table="shuffled")
     G = 2
-    for c in range(2):
+    for c in range(Hkv):
         for b in range(3):
             w.q[b, c * G:(c + 1) * G] = w.q[b, c * G]
     def set_logit(b, toks, target):
-        for c in range(2):
+        for c in range(Hkv):
             qv = wl.bf16_bits_to_f64(w.q[b, c * G])
             k = qv * (target * np.sqrt(128.0) / (qv @ qv))
             for i in toks:
@@ -212,21 +221,23 @@ def test_combine_on_handmade_states():
 @pytest.mark.parametrize("flags", KERNELS)
 @pytest.mark.parametrize("G,seed", [(2, 0), (4, 1), (8, 2), (1, 3)])
 def test_medium_ragged_batch(G, seed, flags):
+    flags, Hkv = flags
     rng = np.random.default_rng(seed)
     lens = rng.integers(1, 6000, size=12).tolist() + [4096, 129, 127]
     ranges = [wl.fixed_shards(L, 1000) for L in lens]
-    w = wl.make_workload("med", lens, ranges, 2 * G, 2, seed=seed, pool_factor=1.2, poison_unused=True,
+    w = wl.make_workload("med", lens, ranges, Hkv * G, Hkv, seed=seed, pool_factor=1.2, poison_unused=True,
                          poison_tails=True)
     dw = run(w, flags)
     T.compare_all(dw, w, tag=f"G={G}")
     assert dw.status() == 0
 
 
-def test_long_single_request_many_segments():
+@pytest.mark.parametrize("Hkv,flags", [(2, 0), (8, 0), (8, qf.QF_FLAG_HEAD_PARALLEL), (16, qf.QF_FLAG_HEAD_PARALLEL)])
+def test_long_single_request_many_segments(Hkv, flags):
     # one request whose single shard is split over every SM by the balanced schedule
-    L = 150_001
-    w = wl.make_workload("long", [L], [[(0, L)]], 4, 2, seed=29)
-    dw = run(w)
+    L = 150_001 if Hkv <= 8 else 40_001
+    w = wl.make_workload("long", [L], [[(0, L)]], 2 * Hkv, Hkv, seed=29)
+    dw = run(w, flags)
     T.compare_all(dw, w)
 
 
@@ -238,6 +249,8 @@ def test_small_configs_elementwise():
         T.compare_all(dw, w, tag=w.name)
         dws = run(w, qf.QF_FLAG_SIMPLE_KERNEL)
         T.compare_all(dws, w, tag=w.name + "/simple")
+        dwh = run(w, qf.QF_FLAG_HEAD_PARALLEL)
+        T.compare_all(dwh, w, tag=w.name + "/headpar")
 
 
 # T9: run-to-run determinism and canaries around the outputs
@@ -267,15 +280,16 @@ def test_determinism_and_no_stray_writes():
 # debug flag: an out-of-range page index is skipped and reported, never a fault
 @pytest.mark.parametrize("flags", KERNELS)
 def test_bad_page_index_is_reported_not_followed(flags):
+    flags, Hkv = flags
     L = 400
-    w = wl.make_workload("bad", [L, L], [[(0, L)], [(0, L)]], 4, 2, seed=31)
+    w = wl.make_workload("bad", [L, L], [[(0, L)], [(0, L)]], 2 * Hkv, Hkv, seed=31)
     good_entry = int(w.block_table[1, 3])
     w.block_table[1, 3] = w.num_pages + 7
     dw = run(w, flags | qf.QF_FLAG_CHECK_BOUNDS)
     assert dw.status() & qf.QF_STATUS_BAD_PAGE
     # request 0 is untouched; request 1 equals the sweep with page 3's tokens left out
     w.block_table[1, 3] = good_entry
-    w2 = wl.make_workload("bad", [L, L], [[(0, L)], [(0, 48), (64, L)]], 4, 2, seed=31)
+    w2 = wl.make_workload("bad", [L, L], [[(0, L)], [(0, 48), (64, L)]], 2 * Hkv, Hkv, seed=31)
     ref = T.oracle_all(w2)
     got = dw.results()
     assert T.out_err(got[3][0], ref[3][0]) < T.ENG_OUT
@@ -303,14 +317,15 @@ def test_full_size_configs_sampled(cfg):
     assert dw.status() == 0
 
 
-def test_many_entries_plan_in_scratch():
+@pytest.mark.parametrize("Hkv,flags", [(2, 0), (8, 0), (8, qf.QF_FLAG_HEAD_PARALLEL)])
+def test_many_entries_plan_in_scratch(Hkv, flags):
     # more (request, shard) pairs than the in-kernel plan holds: the separate plan kernel path
     rng = np.random.default_rng(41)
     B = 700
     lens = rng.integers(0, 300, size=B).tolist()
     ranges = [wl.even_shards(L, 3) + [(0, 0)] for L in lens]   # S = 4 -> 2,800 entries
-    w = wl.make_workload("many", lens, ranges, 4, 2, seed=41, poison_tails=True)
+    w = wl.make_workload("many", lens, ranges, 2 * Hkv, Hkv, seed=41, poison_tails=True)
     assert w.batch * w.max_shards > 2048
-    dw = run(w)
+    dw = run(w, flags)
     T.compare_all(dw, w)
     assert dw.status() == 0
