@@ -278,6 +278,18 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             }
             e = lo;
         }
+        // Per-segment metadata is kept off the critical path: a shard's token range and the first batch
+        // of its block-table row are the same for all KV heads of the shard, so they are cached in
+        // registers; the next non-empty shard's are fetched one segment ahead.
+        int cur_e = -1, beg = 0, end = 0;
+        int nxt_e = -1, nxt_r0 = 0, nxt_r1 = 0, nxt_len = 0;   // raw range of the next non-empty shard
+        int head_tbl_e = -1, head_tbl = 0;                     // table entries of pages [first_page, +32) of a shard
+        int nxt_tbl_e = -1, nxt_tbl = 0;
+        auto load_tbl = [&](int b_, int page0_, int last_page_) -> int {
+            const long long rb = (long long)b_ * P.max_pages_per_req;
+            const int lp = min(page0_ + lane, last_page_);
+            return block_table ? block_table[rb + lp] : (int)(rb + lp);
+        };
         while (ok && pos < pos1) {
             while (prefix[e + 1] <= pos) ++e;  // skip empty entries
             const int base = prefix[e];
@@ -286,15 +298,28 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             const int c = r / nunits, j = r - c * nunits;
             const int seg_len = min(nunits - j, pos1 - pos);
             const int b = e / S;
-            int beg, end;
-            clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[b], beg, end);
+            if (e != cur_e) {
+                if (e == nxt_e) clamp_range(nxt_r0, nxt_r1, nxt_len, beg, end);
+                else clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[b], beg, end);
+                cur_e = e;
+                if (e == nxt_tbl_e) { head_tbl = nxt_tbl; head_tbl_e = e; }
+                // start fetching the next non-empty shard's range; it is consumed a segment later
+                int e2 = e + 1;
+                while (e2 < n_entries && prefix[e2 + 1] == prefix[e2]) ++e2;
+                nxt_e = -1;
+                if (e2 < n_entries && prefix[e2] < pos1) {
+                    nxt_e = e2;
+                    nxt_r0 = shard_ranges[2 * e2];
+                    nxt_r1 = shard_ranges[2 * e2 + 1];
+                    nxt_len = seq_lens[e2 / S];
+                }
+            }
             const int first_page = beg >> 4, last_page = (end - 1) >> 4;
             // the CTAs whose slices touch this unit: one segment each
             const int p0 = base + c * nunits;
             const int first_cta = p0 / per_cta, last_cta = (p0 + nunits - 1) / per_cta;
             const int nseg = last_cta - first_cta + 1;
             const int first_slot = e * Hkv + c + first_cta;
-            const long long row_base = (long long)b * P.max_pages_per_req;
 
             // table entries are fetched 32 pages at a time
             int tbl_page0 = 0, tbl = 0;
@@ -303,8 +328,19 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                 const int np = min(kPagesPerStage, last_page + 1 - page0);
                 if ((u & (32 / kPagesPerStage - 1)) == 0) {
                     tbl_page0 = page0;
-                    const int lp = min(page0 + lane, last_page);
-                    tbl = block_table ? block_table[row_base + lp] : (int)(row_base + lp);
+                    if (j + u == 0 && head_tbl_e == e) {
+                        tbl = head_tbl;           // the shard's first pages: same for every KV head
+                    } else {
+                        tbl = load_tbl(b, page0, last_page);
+                        if (j + u == 0) { head_tbl = tbl; head_tbl_e = e; }
+                    }
+                }
+                if (u == 1 && nxt_e >= 0 && nxt_tbl_e != nxt_e) {
+                    // the next shard's range has arrived by now: fetch its first table entries too
+                    int nb, ne;
+                    clamp_range(nxt_r0, nxt_r1, nxt_len, nb, ne);
+                    nxt_tbl = load_tbl(nxt_e / S, nb >> 4, (ne - 1) >> 4);
+                    nxt_tbl_e = nxt_e;
                 }
                 const int i = lane % kPagesPerStage;    // page within the stage
                 const int part = lane / kPagesPerStage; // 0: K page, 1: V page (>= 2: idle lane)
