@@ -185,9 +185,9 @@ int qf_combine(const float *o_part, const float *lse_part, const int32_t *shard_
     if (rc != QF_OK) return rc;
     const long long bh = (long long)p->batch * p->num_q_heads;
     const unsigned blocks = (unsigned)((bh + qf::kCombineWarps - 1) / qf::kCombineWarps);
-    qf::combine_kernel<<<blocks, qf::kCombineWarps * 32, 0, (cudaStream_t)cuda_stream>>>(
-        o_part, lse_part, shard_counts, out, lse, p->batch, p->num_q_heads, p->max_shards);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = qf::launch_pdl(qf::combine_kernel, dim3(blocks), dim3(qf::kCombineWarps * 32), 0,
+                                   (cudaStream_t)cuda_stream, o_part, lse_part, shard_counts, out, lse, p->batch,
+                                   p->num_q_heads, p->max_shards);
     if (e != cudaSuccess) return cuda_fail(e, "combine_kernel launch");
     g_last_launches = 1;
     return QF_OK;

@@ -15,6 +15,8 @@ combine_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_p
                const int *__restrict__ shard_counts, float *__restrict__ out, float *__restrict__ lse,
                int batch, int num_q_heads, int max_shards)
 {
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int lane = threadIdx.x & 31;
     const long long bh = (long long)blockIdx.x * kCombineWarps + (threadIdx.x >> 5);
     if (bh >= (long long)batch * num_q_heads) return;

@@ -28,6 +28,13 @@ struct DevParams {
     float sm_scale;
 };
 
+// Programmatic dependent launch: every kernel of the path is launched with the programmatic-stream-
+// serialization attribute, so its CTAs may become resident while the previous kernel of the stream is
+// still draining.  grid_dependency_wait() returns once that previous kernel has completed and its
+// writes are visible: it precedes the first global read or write of every kernel.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000u); }
 
 // bf16 pair packed in a 32-bit word -> two fp32 (exact).
@@ -76,6 +83,24 @@ __device__ __forceinline__ void clamp_range(int r0, int r1, int len, int &beg, i
     beg = max(r0, 0);
     end = min(r1, len);
     if (end < beg) end = beg;
+}
+
+// Launch with the programmatic-stream-serialization attribute (see grid_dependency_wait).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 }  // namespace qf

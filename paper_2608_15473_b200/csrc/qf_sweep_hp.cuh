@@ -120,8 +120,10 @@ sweep_hp_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if (blockIdx.x == 0) header[kHdrLastEpoch] = epoch;
     }
+    grid_dependency_wait();     // nothing above touches global memory
+    grid_launch_dependents();
+    if (blockIdx.x == 0 && tid == 0) header[kHdrLastEpoch] = epoch;
 
     // ---- plan: prefix sum of pages x head groups over (request, shard) entries
     const int *prefix;
@@ -417,10 +419,9 @@ int launch_sweep_hp_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const vo
         *launches += 1;
     }
     if (ev0) cudaEventRecord(ev0, st);
-    sweep_hp_kernel<G><<<n_ctas, kSweepThreads, smem, st>>>(kmap, vmap, (const uint16_t *)q, bt, sl, sr, o, m, l,
-                                                             header, global_prefix, counters, seg, wsl.seg_stride,
-                                                             epoch, P);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(sweep_hp_kernel<G>, dim3(n_ctas), dim3(kSweepThreads), smem, st, kmap, vmap,
+                               (const uint16_t *)q, bt, sl, sr, o, m, l, header, global_prefix, counters, seg,
+                               wsl.seg_stride, epoch, P);
     if (ev1) cudaEventRecord(ev1, st);
     if (e != cudaSuccess) { snprintf(msg, msg_len, "sweep_hp_kernel launch: %s", cudaGetErrorString(e)); return -5; }
     *launches += 1;
