@@ -336,3 +336,50 @@ int qfo_combine_fold(const double *o_part, const double *lse_part, const int32_t
     }
     return 0;
 }
+
+/*
+ * The accelerator-side finish of a decode step (Section 2; the fold of the
+ * appendix's "what the combine is"): the cached positions act as one pseudo-token
+ * of score lse_prev and value o_prev, and the current token (k_new, v_new) is
+ * appended to it:
+ *     s_jj = q . k_new / sqrt(d)
+ *     out  = lerp(v_new, o_prev, sigma(lse_prev - s_jj)),  lerp(x,y,t) = (1-t)x + ty
+ *     lse  = logaddexp(lse_prev, s_jj)
+ * with sigma(x) = 1/(1+e^{-x}).  An empty cache (lse_prev = -inf) gives out = v_new,
+ * lse = s_jj.  Query head h uses the new key/value of KV head h / G.
+ *   o_prev [B][Hq][D], lse_prev [B][Hq] (fp64); q [B][Hq][D], k_new/v_new [B][Hkv][D] (bf16 bits)
+ *   out [B][Hq][D], lse [B][Hq], s_self [B][Hq] (optional)
+ */
+int qfo_self_fold(const double *o_prev, const double *lse_prev, const uint16_t *q, const uint16_t *k_new,
+                  const uint16_t *v_new, const qfo_shape *sh, double *out, double *lse, double *s_self)
+{
+    const int B = sh->batch, H = sh->num_q_heads, D = sh->head_dim;
+    if (sh->num_q_heads % sh->num_kv_heads) return -1;
+    const int G = H / sh->num_kv_heads;
+    const double scale = scale_of(sh);
+    for (int b = 0; b < B; ++b) {
+        for (int h = 0; h < H; ++h) {
+            const int c = h / G;
+            const uint16_t *qr = q + ((int64_t)b * H + h) * D;
+            const uint16_t *kr = k_new + ((int64_t)b * sh->num_kv_heads + c) * D;
+            const uint16_t *vr = v_new + ((int64_t)b * sh->num_kv_heads + c) * D;
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d) dot += bf16_to_f64(qr[d]) * bf16_to_f64(kr[d]);
+            const double sjj = dot * scale;
+            const double lp = lse_prev[(int64_t)b * H + h];
+            double *o = out + ((int64_t)b * H + h) * D;
+            const double *op = o_prev + ((int64_t)b * H + h) * D;
+            if (s_self) s_self[(int64_t)b * H + h] = sjj;
+            if (lp == -INFINITY) {
+                for (int d = 0; d < D; ++d) o[d] = bf16_to_f64(vr[d]);
+                lse[(int64_t)b * H + h] = sjj;
+                continue;
+            }
+            const double t = sigmoid(lp - sjj);
+            for (int d = 0; d < D; ++d) o[d] = (1.0 - t) * bf16_to_f64(vr[d]) + t * op[d];
+            lse[(int64_t)b * H + h] = logaddexp(lp, sjj);
+        }
+    }
+    return 0;
+}
+

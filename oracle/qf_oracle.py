@@ -198,3 +198,18 @@ def combine_fold(o_part, lse_part, shard_counts, sh: Shape, perm=None):
                                 _p(out, np.float64), _p(lse, np.float64))
     assert rc == 0
     return out, lse
+
+
+def self_fold(o_prev, lse_prev, q, k_new, v_new, sh: Shape):
+    """Fold the current token into the swept state: out [B,Hq,D], lse [B,Hq], s_self [B,Hq]."""
+    out = np.zeros((sh.batch, sh.num_q_heads, sh.head_dim), np.float64)
+    lse = np.zeros((sh.batch, sh.num_q_heads), np.float64)
+    s_self = np.zeros((sh.batch, sh.num_q_heads), np.float64)
+    shc = sh.c()
+    rc = lib().qfo_self_fold(_p(np.ascontiguousarray(o_prev), np.float64),
+                             _p(np.ascontiguousarray(lse_prev), np.float64), _p(q, np.uint16),
+                             _p(k_new, np.uint16), _p(v_new, np.uint16), ctypes.byref(shc),
+                             _p(out, np.float64), _p(lse, np.float64), _p(s_self, np.float64))
+    assert rc == 0
+    return out, lse, s_self
+

@@ -414,3 +414,72 @@ def test_lse_statistics_of_the_normal_workload():
     _, lse = full(w)
     qn = (wl.bf16_bits_to_f64(w.q[0]) ** 2).sum(axis=1)
     assert np.abs(lse[0] - (math.log(L) + qn / 256.0)).max() < 0.2
+
+
+# ------------------------------------------------- the current token's fold (Section 2)
+def _with_appended_token(w, k_new, v_new):
+    """A copy of the workload whose cache holds one more position per request: (k_new, v_new)."""
+    lens = [int(L) + 1 for L in w.seq_lens]
+    w2 = wl.make_workload("app", lens, [[(0, L)] for L in lens], w.num_q_heads, w.num_kv_heads, seed=0,
+                          table="identity")
+    for b, L in enumerate(w.seq_lens):
+        for i in range(int(L)):
+            w2.k_cache[w2.block_table[b, i // 16], :, i % 16] = w.k_cache[w.block_table[b, i // 16], :, i % 16]
+            w2.v_cache[w2.block_table[b, i // 16], :, i % 16] = w.v_cache[w.block_table[b, i // 16], :, i % 16]
+        L = int(L)
+        w2.k_cache[w2.block_table[b, L // 16], :, L % 16] = k_new[b]
+        w2.v_cache[w2.block_table[b, L // 16], :, L % 16] = v_new[b]
+    w2.q[:] = w.q
+    return w2
+
+
+def test_self_fold_equals_attention_over_one_more_position():
+    lens = [0, 1, 15, 16, 100]
+    w = wl.make_workload("fold1", lens, [[(0, L)] for L in lens], 8, 2, seed=51)
+    rng = np.random.default_rng(51)
+    k_new = wl.f32_to_bf16_bits(rng.standard_normal((len(lens), 2, 128)).astype(np.float32))
+    v_new = wl.f32_to_bf16_bits(rng.standard_normal((len(lens), 2, 128)).astype(np.float32))
+    sh = shape_of(w)
+    o_prev, lse_prev = full(w)
+    out, lse, s_self = orc.self_fold(o_prev, lse_prev, w.q, k_new, v_new, sh)
+    ref_out, ref_lse = full(_with_appended_token(w, k_new, v_new))
+    assert np.allclose(out, ref_out, rtol=1e-12, atol=1e-14)
+    assert np.allclose(lse, ref_lse, rtol=1e-13, atol=1e-13)
+    # empty cache: the step returns the new value and its own score
+    assert np.array_equal(out[0], wl.bf16_bits_to_f64(v_new[0]).repeat(4, axis=0))
+    assert np.array_equal(lse[0], s_self[0])
+
+
+def test_self_fold_sign_is_not_one_directional():
+    # at cache length one the new score may exceed the cached log-sum-exp by many nats, or fall far below it
+    w = wl.make_workload("fold2", [1, 1], [[(0, 1)], [(0, 1)]], 2, 1, seed=53)
+    qv = wl.bf16_bits_to_f32(w.q)
+    k_new = np.stack([wl.f32_to_bf16_bits(qv[0, :1] * np.float32(1.0)),      # s_jj = |q|^2/sqrt(d) >> lse_prev
+                      wl.f32_to_bf16_bits(qv[1, :1] * np.float32(-1.0))])    # s_jj << lse_prev
+    v_new = wl.f32_to_bf16_bits(np.ones((2, 1, 128), np.float32) * np.float32(3.0))
+    sh = shape_of(w)
+    o_prev, lse_prev = full(w)
+    out, lse, s_self = orc.self_fold(o_prev, lse_prev, w.q, k_new, v_new, sh)
+    assert s_self[0, 0] - lse_prev[0, 0] > 5 and s_self[1, 0] - lse_prev[1, 0] < -5
+    for b in range(2):
+        for h in range(2):
+            t = 1.0 / (1.0 + math.exp(-(lse_prev[b, h] - s_self[b, h])))
+            assert np.allclose(out[b, h], (1 - t) * 3.0 + t * o_prev[b, h], rtol=1e-13)
+            assert lse[b, h] == pytest.approx(np.logaddexp(lse_prev[b, h], s_self[b, h]), rel=1e-14)
+    assert np.abs(out[0, 0] - 3.0).max() < 0.1             # head 0 attends to what just arrived
+    assert np.abs(out[1, 0] - o_prev[1, 0]).max() < 0.1    # head 0 attends to what it already had
+
+
+def test_self_fold_large_magnitudes():
+    # lse_prev = 100 and s_jj = 100: log(e^a + e^b) overflows in fp32, the fold does not
+    o_prev = np.zeros((1, 1, 128)); o_prev[0, 0, 0] = 1.0
+    lse_prev = np.array([[100.0]])
+    q = np.zeros((1, 1, 128), np.uint16); k = np.zeros((1, 1, 128), np.uint16)
+    q[0, 0, 0] = wl.f32_to_bf16_bits(np.float32(100.0)).item()
+    k[0, 0, 0] = wl.f32_to_bf16_bits(np.float32(math.sqrt(128.0))).item()   # bf16(11.3125): s_jj = 99.99...
+    v = wl.f32_to_bf16_bits(np.full((1, 1, 128), 2.0, np.float32))
+    sh = orc.Shape(batch=1, num_q_heads=1, num_kv_heads=1)
+    out, lse, s_self = orc.self_fold(o_prev, lse_prev, q, k, v, sh)
+    assert abs(s_self[0, 0] - 100.0) < 0.05
+    assert lse[0, 0] == pytest.approx(np.logaddexp(100.0, s_self[0, 0]), rel=1e-15) and np.isfinite(out).all()
+    assert abs(out[0, 0, 1] - 1.0) < 0.02   # about half of v = 2 in the channels where o_prev is 0
