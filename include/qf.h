@@ -166,6 +166,33 @@ int qf_combine(const float *o_part, const float *lse_part, const int32_t *shard_
                const qf_params *p, void *cuda_stream);
 
 /*
+ * Section 2, the finish of a decode step: the shard merge of qf_combine with the
+ * current token folded in.  With s_jj = q.k_j/sqrt(d) for the token's own key
+ * and value (k_new, v_new: bf16 [B, Hkv, D]; head h uses KV head h/G),
+ *     out = lerp(v_j, o_<j, sigma(lse_<j - s_jj)),  lse = logaddexp(lse_<j, s_jj),
+ * computed as one more operand (log Z = s_jj, vector v_j) of the max-subtracted
+ * merge, which is the same numbers and is safe for either sign of lse_<j - s_jj
+ * and for an empty cache (out = v_j, lse = s_jj).  q: bf16 [B, Hq, D].  All
+ * pointers are device pointers, 8-byte aligned; shard_counts may be NULL.
+ */
+int qf_combine_self(const float *o_part, const float *lse_part, const int32_t *shard_counts,
+                    const void *q, const void *k_new, const void *v_new,
+                    float *out, float *lse,
+                    const qf_params *p, void *cuda_stream);
+
+/*
+ * Section 2, the cache write nothing waits on: stores the current token's key
+ * and value (bf16 [B, Hkv, D]) at position seq_lens[b] of every request, in the
+ * page block_table[b][seq_lens[b]/16] (identity table if NULL).  seq_lens is
+ * not modified: the caller advances it when the next step begins.  A request
+ * whose position has no allocated page (entry outside [0, num_pages), or past
+ * max_pages_per_req) is skipped.  All pointers are device pointers.
+ */
+int qf_append_kv(void *k_cache, void *v_cache, const int32_t *block_table, const int32_t *seq_lens,
+                 const void *k_new, const void *v_new,
+                 const qf_params *p, void *cuda_stream);
+
+/*
  * One whole decode step driven from HOST buffers, as a serving loop calls it:
  * the query and the step's metadata are copied host -> device, the sweep and
  * the merge run, and the result is copied device -> host.  The KV cache stays

@@ -38,6 +38,7 @@ EXPORTS = (
     "qf_version", "qf_strerror", "qf_workspace_bytes", "qf_decode_partial", "qf_combine",
     "qf_step_scratch_bytes", "qf_decode_step_host", "qf_read_status", "qf_last_launch_count",
     "qf_set_profile_events", "qf_decode_partial_static", "qf_static_scratch_error",
+    "qf_combine_self", "qf_append_kv",
 )
 
 
@@ -95,6 +96,10 @@ def lib() -> ctypes.CDLL:
         L.qf_last_launch_count.restype = ctypes.c_int
         L.qf_set_profile_events.restype = ctypes.c_int
         L.qf_set_profile_events.argtypes = [vp, vp]
+        L.qf_combine_self.restype = ctypes.c_int
+        L.qf_combine_self.argtypes = [vp, vp, i32p, vp, vp, vp, vp, vp, pp, vp]
+        L.qf_append_kv.restype = ctypes.c_int
+        L.qf_append_kv.argtypes = [vp, vp, i32p, i32p, vp, vp, pp, vp]
         L.qf_decode_partial_static.restype = ctypes.c_int
         L.qf_decode_partial_static.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, vp, vp, pp, vp]
         L.qf_static_scratch_error.restype = ctypes.c_char_p
@@ -182,6 +187,26 @@ def combine(o_part, lse_part, shard_counts, out, lse, p: QFParams, stream=None, 
                           ctypes.byref(p), _stream(stream))
     if check and rc != QF_OK:
         raise QFError(rc, "qf_combine")
+    return rc
+
+
+def combine_self(o_part, lse_part, shard_counts, q, k_new, v_new, out, lse, p: QFParams, stream=None,
+                 check: bool = True) -> int:
+    """Shard merge with the current token (k_new, v_new) folded in."""
+    rc = lib().qf_combine_self(_ptr(o_part), _ptr(lse_part), _ptr(shard_counts), _ptr(q), _ptr(k_new),
+                               _ptr(v_new), _ptr(out), _ptr(lse), ctypes.byref(p), _stream(stream))
+    if check and rc != QF_OK:
+        raise QFError(rc, "qf_combine_self")
+    return rc
+
+
+def append_kv(k_cache, v_cache, block_table, seq_lens, k_new, v_new, p: QFParams, stream=None,
+              check: bool = True) -> int:
+    """Write the current token's key and value at position seq_lens[b] of every request."""
+    rc = lib().qf_append_kv(_ptr(k_cache), _ptr(v_cache), _ptr(block_table), _ptr(seq_lens), _ptr(k_new),
+                            _ptr(v_new), ctypes.byref(p), _stream(stream))
+    if check and rc != QF_OK:
+        raise QFError(rc, "qf_append_kv")
     return rc
 
 

@@ -174,8 +174,10 @@ int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache, c
     return rc;
 }
 
-int qf_combine(const float *o_part, const float *lse_part, const int32_t *shard_counts, float *out, float *lse,
-               const qf_params *p, void *cuda_stream)
+namespace {
+int launch_combine(const float *o_part, const float *lse_part, const int32_t *shard_counts, const void *q,
+                   const void *k_new, const void *v_new, float *out, float *lse, const qf_params *p,
+                   void *cuda_stream)
 {
     g_last_launches = 0;
     int rc = validate(p);
@@ -183,12 +185,52 @@ int qf_combine(const float *o_part, const float *lse_part, const int32_t *shard_
     if (!o_part || !lse_part || !out || !lse) return QF_ERR_NULL;
     rc = check_device(nullptr);
     if (rc != QF_OK) return rc;
+    const qf::DevParams P = dev_params(p);
     const long long bh = (long long)p->batch * p->num_q_heads;
     const unsigned blocks = (unsigned)((bh + qf::kCombineWarps - 1) / qf::kCombineWarps);
     cudaError_t e = qf::launch_pdl(qf::combine_kernel, dim3(blocks), dim3(qf::kCombineWarps * 32), 0,
-                                   (cudaStream_t)cuda_stream, o_part, lse_part, shard_counts, out, lse, p->batch,
-                                   p->num_q_heads, p->max_shards);
+                                   (cudaStream_t)cuda_stream, o_part, lse_part, shard_counts, (const uint16_t *)q,
+                                   (const uint16_t *)k_new, (const uint16_t *)v_new, out, lse, p->batch,
+                                   p->num_q_heads, p->num_kv_heads, p->max_shards, P.sm_scale);
     if (e != cudaSuccess) return cuda_fail(e, "combine_kernel launch");
+    g_last_launches = 1;
+    return QF_OK;
+}
+}  // namespace
+
+int qf_combine(const float *o_part, const float *lse_part, const int32_t *shard_counts, float *out, float *lse,
+               const qf_params *p, void *cuda_stream)
+{
+    return launch_combine(o_part, lse_part, shard_counts, nullptr, nullptr, nullptr, out, lse, p, cuda_stream);
+}
+
+int qf_combine_self(const float *o_part, const float *lse_part, const int32_t *shard_counts, const void *q,
+                    const void *k_new, const void *v_new, float *out, float *lse, const qf_params *p,
+                    void *cuda_stream)
+{
+    if (!q || !k_new || !v_new) return QF_ERR_NULL;
+    if (((uintptr_t)q & 7) || ((uintptr_t)k_new & 7) || ((uintptr_t)v_new & 7)) return QF_ERR_BAD_SHAPE;
+    return launch_combine(o_part, lse_part, shard_counts, q, k_new, v_new, out, lse, p, cuda_stream);
+}
+
+int qf_append_kv(void *k_cache, void *v_cache, const int32_t *block_table, const int32_t *seq_lens,
+                 const void *k_new, const void *v_new, const qf_params *p, void *cuda_stream)
+{
+    g_last_launches = 0;
+    int rc = validate(p);
+    if (rc != QF_OK) return rc;
+    if (!k_cache || !v_cache || !seq_lens || !k_new || !v_new) return QF_ERR_NULL;
+    if (((uintptr_t)k_cache & 7) || ((uintptr_t)v_cache & 7) || ((uintptr_t)k_new & 7) || ((uintptr_t)v_new & 7))
+        return QF_ERR_BAD_SHAPE;
+    rc = check_device(nullptr);
+    if (rc != QF_OK) return rc;
+    const qf::DevParams P = dev_params(p);
+    const long long bc = (long long)p->batch * p->num_kv_heads;
+    const unsigned blocks = (unsigned)((bc + qf::kCombineWarps - 1) / qf::kCombineWarps);
+    cudaError_t e = qf::launch_pdl(qf::append_kv_kernel, dim3(blocks), dim3(qf::kCombineWarps * 32), 0,
+                                   (cudaStream_t)cuda_stream, (uint16_t *)k_cache, (uint16_t *)v_cache, block_table,
+                                   seq_lens, (const uint16_t *)k_new, (const uint16_t *)v_new, P);
+    if (e != cudaSuccess) return cuda_fail(e, "append_kv_kernel launch");
     g_last_launches = 1;
     return QF_OK;
 }

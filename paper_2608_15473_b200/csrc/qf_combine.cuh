@@ -2,6 +2,11 @@
 // lerp / sigma / logaddexp combine.  One warp per (request, query head); each
 // lane owns four channels, so a shard's 512-byte vector is one coalesced read.  A slot whose
 // log Z is -inf contributes through a select, never a multiply, so garbage in it is harmless.
+//
+// With a current token (Section 2: s_jj = q.k_j/sqrt(d), out = lerp(v_j, o_<j, sigma(lse_<j - s_jj)),
+// lse = logaddexp(lse_<j, s_jj)) the token is simply one more operand of the same merge, with
+// log Z = s_jj and vector v_j: the two-way lerp/sigma form and the max-subtracted form are the
+// same numbers, and the latter needs no case split on the sign of lse_<j - s_jj.
 #pragma once
 
 #include "qf_common.cuh"
@@ -10,10 +15,13 @@ namespace qf {
 
 constexpr int kCombineWarps = 4;
 
+// q, k_new, v_new: nullptr = no current token.  k_new, v_new: bf16 [B, Hkv, D].
 __global__ void __launch_bounds__(kCombineWarps * 32)
 combine_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_part,
-               const int *__restrict__ shard_counts, float *__restrict__ out, float *__restrict__ lse,
-               int batch, int num_q_heads, int max_shards)
+               const int *__restrict__ shard_counts, const uint16_t *__restrict__ q,
+               const uint16_t *__restrict__ k_new, const uint16_t *__restrict__ v_new,
+               float *__restrict__ out, float *__restrict__ lse,
+               int batch, int num_q_heads, int num_kv_heads, int max_shards, float sm_scale)
 {
     grid_dependency_wait();
     grid_launch_dependents();
@@ -24,9 +32,28 @@ combine_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_p
     int ns = shard_counts ? shard_counts[b] : max_shards;
     ns = min(max(ns, 0), max_shards);
 
+    // the current token, if any: its score against this head's query and its value row
+    float s_self = neg_inf();
+    float4 v_self = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (q != nullptr) {
+        const int c = h / (num_q_heads / num_kv_heads);
+        const uint2 qw = *reinterpret_cast<const uint2 *>(q + (size_t)bh * kHeadDim + lane * 4);
+        const size_t row = ((size_t)b * num_kv_heads + c) * kHeadDim + lane * 4;
+        const uint2 kw = *reinterpret_cast<const uint2 *>(k_new + row);
+        const uint2 vw = *reinterpret_cast<const uint2 *>(v_new + row);
+        float d = bf16lo_to_f32(qw.x) * bf16lo_to_f32(kw.x);
+        d = fmaf(bf16hi_to_f32(qw.x), bf16hi_to_f32(kw.x), d);
+        d = fmaf(bf16lo_to_f32(qw.y), bf16lo_to_f32(kw.y), d);
+        d = fmaf(bf16hi_to_f32(qw.y), bf16hi_to_f32(kw.y), d);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+        s_self = d * sm_scale;
+        v_self = make_float4(bf16lo_to_f32(vw.x), bf16hi_to_f32(vw.x), bf16lo_to_f32(vw.y), bf16hi_to_f32(vw.y));
+    }
+
     const float *lrow = lse_part + ((size_t)b * max_shards) * num_q_heads + h;
-    // M = max over shards of log Z; lanes stride over shards
-    float M = neg_inf();
+    // M = max over operands of log Z; lanes stride over shards
+    float M = s_self;
     for (int s = lane; s < ns; s += 32) M = fmaxf(M, lrow[(size_t)s * num_q_heads]);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
@@ -66,11 +93,44 @@ combine_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_p
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, off);
+        if (s_self != neg_inf()) {
+            const float w = expf(s_self - M);
+            wsum += w;
+            acc.x = fmaf(w, v_self.x, acc.x);
+            acc.y = fmaf(w, v_self.y, acc.y);
+            acc.z = fmaf(w, v_self.z, acc.z);
+            acc.w = fmaf(w, v_self.w, acc.w);
+        }
         const float inv = 1.f / wsum;
         acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
     }
     *reinterpret_cast<float4 *>(out + (size_t)bh * kHeadDim + lane * 4) = acc;
     if (lane == 0) lse[bh] = (M == neg_inf()) ? neg_inf() : M + logf(wsum);
+}
+
+// The cache write nothing waits on (Section 2): the current token's key and value go to position
+// seq_lens[b] of request b, through the block table.  One warp per (request, KV head).
+__global__ void __launch_bounds__(kCombineWarps * 32)
+append_kv_kernel(uint16_t *__restrict__ k_cache, uint16_t *__restrict__ v_cache,
+                 const int *__restrict__ block_table, const int *__restrict__ seq_lens,
+                 const uint16_t *__restrict__ k_new, const uint16_t *__restrict__ v_new, DevParams P)
+{
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const int lane = threadIdx.x & 31;
+    const long long bc = (long long)blockIdx.x * kCombineWarps + (threadIdx.x >> 5);
+    if (bc >= (long long)P.batch * P.num_kv_heads) return;
+    const int b = (int)(bc / P.num_kv_heads), c = (int)(bc % P.num_kv_heads);
+    const int pos = seq_lens[b];
+    const int lp = pos >> 4;
+    if (pos < 0 || lp >= P.max_pages_per_req) return;   // no page for this position: nothing is written
+    const long long phys = block_table ? (long long)block_table[(size_t)b * P.max_pages_per_req + lp]
+                                       : (long long)b * P.max_pages_per_req + lp;
+    if (phys < 0 || phys >= P.num_pages) return;         // unallocated page: nothing is written
+    const size_t dst = (((size_t)phys * P.num_kv_heads + c) * kPageSize + (pos & 15)) * kHeadDim + lane * 4;
+    const size_t src = (size_t)bc * kHeadDim + lane * 4;
+    *reinterpret_cast<uint2 *>(k_cache + dst) = *reinterpret_cast<const uint2 *>(k_new + src);
+    *reinterpret_cast<uint2 *>(v_cache + dst) = *reinterpret_cast<const uint2 *>(v_new + src);
 }
 
 }  // namespace qf
