@@ -31,6 +31,9 @@ if str(ROOT) not in sys.path:
     sys.path.insert(0, str(ROOT))
 
 METRIC = "decode-attention KV GB/s and % of B200 HBM peak (Qwen3-4B shape, batched)"
+# dram__bytes_read.sum + dram__bytes_write.sum of one sweep-kernel launch, from the ncu captures summarised in
+# profiles/sweep_kernel_cfg3_ncu.md and profiles/sweep_kernel_cfg4_traffic.md (seed 0)
+NCU_TRAFFIC_BYTES = {3: 2014590000 + 8948224, 4: 4297704192 + 642816}
 FALLBACK_HBM_GBS = 6650.0
 DATASHEET_HBM_GBS = 8000.0
 
@@ -256,23 +259,17 @@ def run_cuda(args):
         hs.step()       # synchronises the stream before returning
     e2e_s = (time.perf_counter() - t0) * args.steps / e2e_steps
 
-    my_bytes = w.algorithmic_bytes()
-    my_tokens = w.swept_tokens()
-    if dist is not None:
-        t = torch.tensor([elapsed_ms, e2e_s * 1e3, sweep_ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, e2e_ms, sweep_ms_max = (float(x) for x in t.tolist())
-        s = torch.tensor([my_bytes, my_tokens], dtype=torch.float64, device=device)
-        dist.all_reduce(s, op=dist.ReduceOp.SUM)
-        tot_bytes, tot_tokens = (float(x) for x in s.tolist())
-    else:
-        e2e_ms, sweep_ms_max = e2e_s * 1e3, sweep_ms
-        tot_bytes, tot_tokens = float(my_bytes), float(my_tokens)
+    from paper_2608_15473_b200.multi import reduce_timings, whole_job_throughput
+    times, counts = reduce_timings({"elapsed": elapsed_ms, "e2e": e2e_s * 1e3, "sweep": sweep_ms},
+                                   {"bytes": float(w.algorithmic_bytes()), "tokens": float(w.swept_tokens())},
+                                   dist, device)
+    elapsed_ms, e2e_ms = times["elapsed"], times["e2e"]
+    tot_bytes, tot_tokens = counts["bytes"], counts["tokens"]
 
     if rank == 0:
         peak, peak_kind = measured_peaks()
         ms_per_step = elapsed_ms / args.steps
-        value = tot_bytes / (ms_per_step * 1e-3) / 1e9
+        value = whole_job_throughput(tot_bytes, ms_per_step)
         kbytes = sweep_kernel_bytes(w)
         achieved = kbytes / (sweep_ms * 1e-3) / 1e9
         line = {
@@ -284,7 +281,7 @@ def run_cuda(args):
                        "l2": "inputs larger than L2 (KV bytes per step >> 126 MB), no flush needed",
                        "parallelism": f"requests sharded over {world} GPU(s), no collective"},
             "clocks": clocks.summary(),
-            "e2e": {"value": tot_bytes / (e2e_ms * 1e-3 / args.steps) / 1e9, "unit": "GB/s",
+            "e2e": {"value": whole_job_throughput(tot_bytes, e2e_ms / args.steps), "unit": "GB/s",
                     "h2d_bytes_per_step": hs.h2d_bytes, "d2h_bytes_per_step": hs.d2h_bytes,
                     "ms_per_step": e2e_ms / args.steps,
                     "note": "qf_decode_step_host: q and step metadata copied in, out and lse copied back; "
@@ -294,7 +291,9 @@ def run_cuda(args):
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "frac_of_datasheet_8TBs": achieved / DATASHEET_HBM_GBS,
                          "ms_per_launch": sweep_ms, "bytes_per_launch": kbytes,
-                         "traffic": args.ncu_traffic},
+                         "traffic": args.ncu_traffic if args.ncu_traffic is not None else
+                         (NCU_TRAFFIC_BYTES.get(args.workload) if args.seed == 0 else None),
+                         "note": "kernel timed by an event pair around each launch in a second K-step region"},
             "kv_tokens_per_s": tot_tokens / (ms_per_step * 1e-3),
             "pct_of_hbm_peak": 100.0 * value / (peak * world),
         }
