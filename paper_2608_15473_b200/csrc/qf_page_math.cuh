@@ -131,19 +131,32 @@ __device__ __forceinline__ void process_page(uint32_t k_base, uint32_t v_base, i
     }
 
     // ---- S[token, head] = K Q^T: A = K tile (row major), B = Q^T fragments
+    // All K fragments are fetched before the first MMA, and the V fragments right after the last one, so
+    // that shared-memory latency overlaps the tensor pipe and the softmax arithmetic below.
     float sc[4] = {0.f, 0.f, 0.f, 0.f};
+    uint32_t vfrag[8][4];
     {
         float sc_odd[4] = {0.f, 0.f, 0.f, 0.f};  // two accumulators: half the dependent-MMA chain
+        uint32_t kfrag[8][4];
         const int row = (lane & 7) + ((lane >> 3) & 1) * 8;
         const int csel = lane >> 4;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             const int chunk = 2 * ks + csel;  // 16-byte chunk of the 256-byte row
-            const uint32_t addr = k_base + (chunk >> 3) * half_stride + row * 128 + (((chunk & 7) ^ (row & 7)) << 4);
-            uint32_t a[4];
-            ldmatrix_x4(a, addr);
-            if (ks & 1) mma_bf16(sc_odd, a, qf[ks][0], qf[ks][1]);
-            else mma_bf16(sc, a, qf[ks][0], qf[ks][1]);
+            ldmatrix_x4(kfrag[ks], k_base + (chunk >> 3) * half_stride + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+        }
+#pragma unroll
+        for (int ks = 0; ks < 8; ks += 2) {
+            mma_bf16(sc, kfrag[ks], qf[ks][0], qf[ks][1]);
+            mma_bf16(sc_odd, kfrag[ks + 1], qf[ks + 1][0], qf[ks + 1][1]);
+        }
+        const int vrow = (lane & 7) + (lane >> 4) * 8;
+        const int vsel = (lane >> 3) & 1;
+#pragma unroll
+        for (int mt_i = 0; mt_i < 8; ++mt_i) {   // A = V^T via transposing loads
+            const int chunk = 2 * mt_i + vsel;
+            ldmatrix_x4_trans(vfrag[mt_i],
+                              v_base + (chunk >> 3) * half_stride + vrow * 128 + (((chunk & 7) ^ (vrow & 7)) << 4));
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) sc[i] += sc_odd[i];
@@ -183,20 +196,12 @@ __device__ __forceinline__ void process_page(uint32_t k_base, uint32_t v_base, i
     const uint32_t bh0 = movmatrix_trans(h0), bh1 = movmatrix_trans(h1);
     const uint32_t bl0 = movmatrix_trans(l0), bl1 = movmatrix_trans(l1);
 
-    // ---- O^T[d, head] += V^T P^T: A = V^T via transposing loads
-    {
-        const int row = (lane & 7) + (lane >> 4) * 8;
-        const int csel = (lane >> 3) & 1;
+    // ---- O^T[d, head] += V^T P^T: the eight hi products first, then the eight lo products, so that no
+    // MMA waits on the one just issued for the same accumulator
 #pragma unroll
-        for (int mt_i = 0; mt_i < 8; ++mt_i) {
-            const int chunk = 2 * mt_i + csel;
-            const uint32_t addr = v_base + (chunk >> 3) * half_stride + row * 128 + (((chunk & 7) ^ (row & 7)) << 4);
-            uint32_t a[4];
-            ldmatrix_x4_trans(a, addr);
-            mma_bf16(acc[mt_i], a, bh0, bh1);
-            mma_bf16(acc[mt_i], a, bl0, bl1);
-        }
-    }
+    for (int mt_i = 0; mt_i < 8; ++mt_i) mma_bf16(acc[mt_i], vfrag[mt_i], bh0, bh1);
+#pragma unroll
+    for (int mt_i = 0; mt_i < 8; ++mt_i) mma_bf16(acc[mt_i], vfrag[mt_i], bl0, bl1);
 }
 
 }  // namespace qf

@@ -37,19 +37,11 @@
 
 namespace qf {
 
-#ifndef QF_PAGES_PER_STAGE
-#define QF_PAGES_PER_STAGE 8
-#endif
-#ifndef QF_STAGES
-#define QF_STAGES (24 / QF_PAGES_PER_STAGE)
-#endif
 constexpr int kConsumerWarps = 8;
-constexpr int kPagesPerStage = QF_PAGES_PER_STAGE;          // pages (of one KV head) per ring stage: 8, 4 or 2
-constexpr int kTeams         = kConsumerWarps / kPagesPerStage;  // warp teams that take stages in turn
+constexpr int kPagesPerStage = kConsumerWarps;    // pages (of one KV head) per ring stage, one per consumer warp
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kSweepThreads  = (kConsumerWarps + 1) * 32;
-constexpr int kStages        = QF_STAGES;
-static_assert(kPagesPerStage == 8 || kPagesPerStage == 4 || kPagesPerStage == 2, "stage must hold 8, 4 or 2 pages");
+constexpr int kStages        = 3;                 // 3 x 64 KB of K and V in flight per SM
 constexpr int kMaxSweepCtas  = 160;               // persistent CTAs (one per SM) are capped at this
 constexpr int kHalfTileBytes = 2048;              // 16 rows x 64 channels of bf16
 constexpr int kRedStride     = kHeadDim + 4;      // padded row of the warp-merge buffer
@@ -422,9 +414,9 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     float m2[2] = {neg_inf(), neg_inf()};
     float l[2] = {0.f, 0.f};
     float acc[8][4];
-    int stage = 0, seq = 0;
+    int stage = 0;
     uint32_t phase = 0, red_phase0 = 0, red_phase1 = 0;
-    const int team = warp / kPagesPerStage, wp = warp % kPagesPerStage;  // teams take stages in turn
+    const int wp = warp;  // this warp's page within a stage
 
     // every consumer warp waits on the warp-merge barriers through this; false = abort
     auto red_sync = [&](int which, uint32_t &ph) -> bool {
@@ -459,13 +451,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             for (int i = 0; i < 8; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
         }
 
-        const bool my_turn = (kTeams == 1) || ((seq % kTeams) == team);
-        ++seq;
-#ifdef QF_EXP_NOCOMPUTE
-        if (false) {
-#else
-        if (my_turn && wp < mt.npages) {
-#endif
+        if (wp < mt.npages) {
             const int tok0 = (mt.page0 + wp) << 4;
             int tlo = max(mt.tok_beg - tok0, 0), thi = min(mt.tok_end - tok0, kPageSize);
             if ((mt.aux >> wp) & 1) { tlo = 0; thi = 0; }

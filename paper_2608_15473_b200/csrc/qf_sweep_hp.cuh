@@ -25,10 +25,7 @@ namespace qf {
 constexpr int kHpHeads = 8;                              // KV heads per stage, one per consumer warp
 constexpr int kHpTileBytes = kHpHeads * kPageBytes;      // 32 KB: K (or V) of one page, eight heads
 constexpr int kHpHalfStride = kHpTileBytes / 2;          // the two 64-channel halves of the box
-#ifndef QF_HP_STAGES
-#define QF_HP_STAGES 3
-#endif
-constexpr int kHpStages = QF_HP_STAGES;
+constexpr int kHpStages = 3;
 
 template <int G>
 struct HpSmem {
