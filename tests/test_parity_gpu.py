@@ -308,7 +308,7 @@ def test_host_step_matches_device_path():
 
 
 # T8: the benchmark configurations at full size, sampled outputs
-@pytest.mark.parametrize("cfg", [2, 3, 4])
+@pytest.mark.parametrize("cfg", [2, 3, 4, 5])
 def test_full_size_configs_sampled(cfg):
     w = wl.CONFIGS[cfg](seed=0)
     dw = run(w)
