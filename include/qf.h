@@ -221,6 +221,18 @@ int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_c
 int qf_read_status(const void *workspace, int32_t *host_status, void *cuda_stream);
 
 /*
+ * Diagnostic aid (no counterpart in the paper).  Every wait inside the kernels
+ * is bounded: when its limit runs out the kernel records QF_STATUS_TIMEOUT and
+ * returns instead of hanging.  This call enqueues a one-warp kernel that waits,
+ * with a limit of a few thousand polls (under a millisecond), on a barrier that
+ * nothing will ever complete, through the same wait routine; afterwards
+ * qf_read_status(workspace) must report QF_STATUS_TIMEOUT and the context must
+ * still be usable.  `workspace`: at least 256 bytes of device memory, 256-byte
+ * aligned (its header words are overwritten).
+ */
+int qf_selftest_bounded_wait(void *workspace, void *cuda_stream);
+
+/*
  * Number of kernels the last qf_decode_partial / qf_combine call on this
  * thread enqueued (for launch accounting in benchmarks).
  */

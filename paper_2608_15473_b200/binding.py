@@ -38,7 +38,7 @@ EXPORTS = (
     "qf_version", "qf_strerror", "qf_workspace_bytes", "qf_decode_partial", "qf_combine",
     "qf_step_scratch_bytes", "qf_decode_step_host", "qf_read_status", "qf_last_launch_count",
     "qf_set_profile_events", "qf_decode_partial_static", "qf_static_scratch_error",
-    "qf_combine_self", "qf_append_kv",
+    "qf_combine_self", "qf_append_kv", "qf_selftest_bounded_wait",
 )
 
 
@@ -100,6 +100,8 @@ def lib() -> ctypes.CDLL:
         L.qf_combine_self.argtypes = [vp, vp, i32p, vp, vp, vp, vp, vp, pp, vp]
         L.qf_append_kv.restype = ctypes.c_int
         L.qf_append_kv.argtypes = [vp, vp, i32p, i32p, vp, vp, pp, vp]
+        L.qf_selftest_bounded_wait.restype = ctypes.c_int
+        L.qf_selftest_bounded_wait.argtypes = [vp, vp]
         L.qf_decode_partial_static.restype = ctypes.c_int
         L.qf_decode_partial_static.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, vp, vp, pp, vp]
         L.qf_static_scratch_error.restype = ctypes.c_char_p
@@ -220,6 +222,13 @@ def decode_step_host(q_host, k_cache, v_cache, block_table, seq_lens_host, shard
     if check and rc != QF_OK:
         raise QFError(rc, "qf_decode_step_host")
     return rc
+
+
+def selftest_bounded_wait(workspace, stream=None) -> None:
+    """Enqueue the kernel whose wait can never be satisfied; read_status must then report a timeout."""
+    rc = lib().qf_selftest_bounded_wait(_ptr(workspace), _stream(stream))
+    if rc != QF_OK:
+        raise QFError(rc, "qf_selftest_bounded_wait")
 
 
 def read_status(workspace, stream=None) -> int:

@@ -311,6 +311,19 @@ int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_c
     return QF_OK;
 }
 
+int qf_selftest_bounded_wait(void *workspace, void *cuda_stream)
+{
+    if (!workspace) return QF_ERR_NULL;
+    if ((uintptr_t)workspace & 255) return QF_ERR_WORKSPACE;
+    int rc = check_device(nullptr);
+    if (rc != QF_OK) return rc;
+    qf::selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)cuda_stream>>>((unsigned long long *)workspace,
+                                                                      qf::next_epoch(), 1u << 12);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "selftest_wait_kernel launch");
+    return QF_OK;
+}
+
 int qf_read_status(const void *workspace, int32_t *host_status, void *cuda_stream)
 {
     if (!workspace || !host_status) return QF_ERR_NULL;

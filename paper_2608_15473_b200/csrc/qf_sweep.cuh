@@ -546,6 +546,25 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     }
 }
 
+// ------------------------------------------------------------------ bounded-wait self-test
+// Waits, with a short limit, on a barrier that nothing will ever complete, through the same wait
+// routine the sweep kernels use: the wait must give up, report QF_STATUS_TIMEOUT and let the kernel
+// return, leaving the context usable.
+__global__ void selftest_wait_kernel(unsigned long long *header, unsigned long long epoch, unsigned limit)
+{
+    __shared__ alignas(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        header[kHdrLastEpoch] = epoch;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && !mbar_wait(smem_u32(&bar), 0, &abort_flag, limit))
+        epoch_or(header + kHdrStatus, epoch, kStatusTimeout);
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,

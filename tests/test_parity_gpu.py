@@ -329,3 +329,15 @@ def test_many_entries_plan_in_scratch(Hkv, flags):
     dw = run(w, flags)
     T.compare_all(dw, w)
     assert dw.status() == 0
+
+
+def test_a_wait_that_cannot_be_satisfied_times_out_and_leaves_the_context_usable():
+    w = wl.config3(seed=9, batch=3, hi=3000)
+    dw = DeviceWorkload(w)
+    qf.selftest_bounded_wait(dw.workspace)
+    assert dw.status() == qf.QF_STATUS_TIMEOUT
+    # the same workspace and context go on working, and the stale status does not leak into the next launch
+    dw.poison_outputs()
+    dw.step()
+    assert dw.status() == 0
+    T.compare_all(dw, w)
