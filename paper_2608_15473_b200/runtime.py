@@ -99,8 +99,16 @@ class HostStepper:
                           self.shard_ranges_host.numel() * 4 + self.shard_counts_host.numel() * 4)
         self.d2h_bytes = self.out_host.numel() * 4 + self.lse_host.numel() * 4
 
+        # raw addresses once: the per-step call then only crosses the C boundary
+        import ctypes
+        self._fn = qf.lib().qf_decode_step_host
+        self._args = [qf._ptr(x) for x in (self.q_host, dw.k_cache, dw.v_cache, dw.block_table, self.seq_lens_host,
+                                           self.shard_ranges_host, self.shard_counts_host, self.out_host,
+                                           self.lse_host)]
+        self._tail = [ctypes.byref(dw.params), qf._ptr(self.scratch), int(self.scratch_bytes)]
+
     def step(self, stream=None) -> None:
-        dw = self.dw
-        qf.decode_step_host(self.q_host, dw.k_cache, dw.v_cache, dw.block_table, self.seq_lens_host,
-                            self.shard_ranges_host, self.shard_counts_host, self.out_host, self.lse_host,
-                            dw.params, self.scratch, self.scratch_bytes, stream)
+        st = int(torch.cuda.current_stream().cuda_stream) if stream is None else qf._stream(stream)
+        rc = self._fn(*self._args, *self._tail, st)
+        if rc != qf.QF_OK:
+            raise qf.QFError(rc, "qf_decode_step_host")
