@@ -50,12 +50,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     return false;
 }
-// One (page, KV head) block: 64 channels x 16 rows x 2 halves = 4 KB in one request.
-__device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap *map, int row, uint32_t bar)
+// L2 policy for the K/V stream: every byte is used once, so its lines should be the first to go and
+// leave the L2 to what is reused (shard states, segment slots, block table, q).
+__device__ __forceinline__ unsigned long long l2_evict_first_policy()
+{
+    unsigned long long policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+// One TMA box (a page of one KV head: 64 channels x 16 rows x 2 halves = 4 KB; or of eight heads: 32 KB).
+__device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap *map, int row, uint32_t bar,
+                                              unsigned long long policy)
 {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(0), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(0), "r"(bar), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
 {

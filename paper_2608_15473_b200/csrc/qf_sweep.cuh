@@ -158,19 +158,39 @@ __device__ __forceinline__ void merge_segments(const float *__restrict__ seg, in
                                                float *__restrict__ m_part, float *__restrict__ lse_part, int tid)
 {
     const float kLn2 = 0.6931471805599453f;
+    constexpr int kBatch = 8;   // segments whose loads are in flight together
     for (int idx = tid; idx < G * kHeadDim; idx += NT) {
         const int head = idx >> 7, d = idx & 127;
         float M = neg_inf();
-        for (int i = 0; i < nseg; ++i)
-            M = fmaxf(M, __ldcg(seg + (size_t)(first_slot + i * slot_step) * seg_stride + G * kHeadDim + 2 * head));
+        for (int base = 0; base < nseg; base += kBatch) {
+            float mv[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u)
+                mv[u] = (base + u < nseg)
+                            ? __ldcg(seg + (size_t)(first_slot + (base + u) * slot_step) * seg_stride + G * kHeadDim + 2 * head)
+                            : neg_inf();
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) M = fmaxf(M, mv[u]);
+        }
         const bool empty = (M == neg_inf());
         const float Ms = empty ? 0.f : M;
         float z = 0.f, wsum = 0.f;
-        for (int i = 0; i < nseg; ++i) {
-            const float *sl = seg + (size_t)(first_slot + i * slot_step) * seg_stride;
-            const float ew = fast_exp2(__ldcg(sl + G * kHeadDim + 2 * head) - Ms);
-            z = fmaf(__ldcg(sl + G * kHeadDim + 2 * head + 1), ew, z);
-            wsum = fmaf(__ldcg(sl + head * kHeadDim + d), ew, wsum);
+        for (int base = 0; base < nseg; base += kBatch) {
+            float mv[kBatch], zv[kBatch], av[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const bool on = base + u < nseg;
+                const float *sl = seg + (size_t)(first_slot + (on ? base + u : 0) * slot_step) * seg_stride;
+                mv[u] = on ? __ldcg(sl + G * kHeadDim + 2 * head) : neg_inf();
+                zv[u] = on ? __ldcg(sl + G * kHeadDim + 2 * head + 1) : 0.f;
+                av[u] = on ? __ldcg(sl + head * kHeadDim + d) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {   // fixed order: deterministic
+                const float ew = fast_exp2(mv[u] - Ms);
+                z = fmaf(zv[u], ew, z);
+                wsum = fmaf(av[u], ew, wsum);
+            }
         }
         o_part[(out_row + head) * kHeadDim + d] = empty ? 0.f : wsum / z;
         if (d == 0) {
@@ -258,6 +278,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
 
     if (warp == kConsumerWarps) {
         // ============================ producer warp ============================
+        const unsigned long long kv_policy = l2_evict_first_policy();
         int stage = 0;
         uint32_t phase = 0;
         int issued = 0;
@@ -360,7 +381,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                 __syncwarp();
                 if (issuer) {
                     const int row = (phys * Hkv + c) * kPageSize;
-                    tma_load_page(smem_u32(&sm.kv[stage][part][i][0]), part ? &v_map : &k_map, row, full);
+                    tma_load_page(smem_u32(&sm.kv[stage][part][i][0]), part ? &v_map : &k_map, row, full, kv_policy);
                 }
                 if (first && lane == 0)
                     bulk_load_1d(smem_u32(&sm.q[stage][0]), q + ((size_t)b * Hq + (size_t)c * G) * kHeadDim,
@@ -494,30 +515,36 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                     }
                 }
                 if (!red_sync(0, red_phase0)) return;
-                for (int idx = tid; idx < RG * kHeadDim; idx += kConsumerThreads) {
-                    const int hl = idx >> 7, d = idx & 127;
+                {
+                    // kThreadsPerHead threads share a head: the eight warps' weights are computed once per thread
+                    constexpr int kThreadsPerHead = kConsumerThreads / RG;
+                    const int hl = tid / kThreadsPerHead, d0 = tid % kThreadsPerHead;
                     const int head = hr * RG + hl;
                     float M = neg_inf();
 #pragma unroll
                     for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm.red_ml[w][head][0]);
-                    const float Ms = (M == neg_inf()) ? 0.f : M;
-                    float z = 0.f, wsum = 0.f;
+                    const bool empty = (M == neg_inf());
+                    const float Ms = empty ? 0.f : M;
+                    float ew[kConsumerWarps];
+                    float z = 0.f;
 #pragma unroll
                     for (int w = 0; w < kConsumerWarps; ++w) {
-                        const float ew = fast_exp2(sm.red_ml[w][head][0] - Ms);
-                        z = fmaf(sm.red_ml[w][head][1], ew, z);
-                        wsum = fmaf(sm.red_acc[w][hl][d], ew, wsum);
+                        ew[w] = fast_exp2(sm.red_ml[w][head][0] - Ms);
+                        z = fmaf(sm.red_ml[w][head][1], ew[w], z);
                     }
-                    if (nseg == 1) {
-                        const bool empty = (M == neg_inf());
-                        o_part[(out_row + head) * kHeadDim + d] = empty ? 0.f : wsum / z;
-                        if (d == 0) {
+                    const float inv = empty ? 0.f : 1.f / z;
+                    for (int d = d0; d < kHeadDim; d += kThreadsPerHead) {
+                        float wsum = 0.f;
+#pragma unroll
+                        for (int w = 0; w < kConsumerWarps; ++w) wsum = fmaf(sm.red_acc[w][hl][d], ew[w], wsum);
+                        if (nseg == 1) o_part[(out_row + head) * kHeadDim + d] = wsum * inv;
+                        else __stcg(seg_slot + head * kHeadDim + d, wsum);
+                    }
+                    if (d0 == 0) {
+                        if (nseg == 1) {
                             m_part[out_row + head] = empty ? neg_inf() : M * kLn2;
                             lse_part[out_row + head] = empty ? neg_inf() : (M + log2f(z)) * kLn2;
-                        }
-                    } else {
-                        __stcg(seg_slot + head * kHeadDim + d, wsum);
-                        if (d == 0) {
+                        } else {
                             __stcg(seg_slot + G * kHeadDim + 2 * head, M);
                             __stcg(seg_slot + G * kHeadDim + 2 * head + 1, z);
                         }

@@ -52,13 +52,6 @@ struct Pieces {
     __device__ __forceinline__ int end(int p) const { return min((p + 1) * qs, total); }
 };
 
-__device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap *map, int row, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(0), "r"(bar) : "memory");
-}
-
 // Merge the segments a (shard, KV head) unit was cut into, pieces p_first .. p_first+nseg-1, in that
 // order (deterministic), by the one warp that arrived last.
 template <int G>
@@ -70,18 +63,37 @@ __device__ __forceinline__ void merge_pieces(const float *__restrict__ seg, int 
     auto slot_of = [&](int i) -> const float * {
         return seg + (size_t)((2 * (p_first + i) + (i == 0 ? 1 : 0)) * kHpHeads + head_in_group) * seg_stride;
     };
+    constexpr int kBatch = 8;   // segments whose loads are in flight together
     for (int idx = lane; idx < G * kHeadDim; idx += 32) {
         const int head = idx >> 7, d = idx & 127;
         float M = neg_inf();
-        for (int i = 0; i < nseg; ++i) M = fmaxf(M, __ldcg(slot_of(i) + G * kHeadDim + 2 * head));
+        for (int base = 0; base < nseg; base += kBatch) {
+            float mv[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u)
+                mv[u] = (base + u < nseg) ? __ldcg(slot_of(base + u) + G * kHeadDim + 2 * head) : neg_inf();
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) M = fmaxf(M, mv[u]);
+        }
         const bool empty = (M == neg_inf());
         const float Ms = empty ? 0.f : M;
         float z = 0.f, wsum = 0.f;
-        for (int i = 0; i < nseg; ++i) {
-            const float *sl = slot_of(i);
-            const float ew = fast_exp2(__ldcg(sl + G * kHeadDim + 2 * head) - Ms);
-            z = fmaf(__ldcg(sl + G * kHeadDim + 2 * head + 1), ew, z);
-            wsum = fmaf(__ldcg(sl + head * kHeadDim + d), ew, wsum);
+        for (int base = 0; base < nseg; base += kBatch) {
+            float mv[kBatch], zv[kBatch], av[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const bool on = base + u < nseg;
+                const float *sl = slot_of(on ? base + u : 0);
+                mv[u] = on ? __ldcg(sl + G * kHeadDim + 2 * head) : neg_inf();
+                zv[u] = on ? __ldcg(sl + G * kHeadDim + 2 * head + 1) : 0.f;
+                av[u] = on ? __ldcg(sl + head * kHeadDim + d) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {   // fixed order: deterministic
+                const float ew = fast_exp2(mv[u] - Ms);
+                z = fmaf(zv[u], ew, z);
+                wsum = fmaf(av[u], ew, wsum);
+            }
         }
         o_part[(out_row + head) * kHeadDim + d] = empty ? 0.f : wsum / z;
         if (d == 0) {
@@ -164,6 +176,7 @@ sweep_hp_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
 
     if (warp == kConsumerWarps) {
         // ============================ producer warp ============================
+        const unsigned long long kv_policy = l2_evict_first_policy();
         int stage = 0;
         uint32_t phase = 0;
         int issued = 0;
@@ -225,7 +238,7 @@ sweep_hp_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 __syncwarp();
                 if (lane < 2) {    // two 32 KB boxes: K and V of the page, eight heads each
                     const int row = (phys * Hkv + grp * kHpHeads) * kPageSize;
-                    tma_load_box(smem_u32(&sm.kv[stage][lane][0]), lane ? &v_map : &k_map, row, full);
+                    tma_load_page(smem_u32(&sm.kv[stage][lane][0]), lane ? &v_map : &k_map, row, full, kv_policy);
                 } else if (lane == 2 && first) {
                     bulk_load_1d(smem_u32(&sm.q[stage][0]),
                                  q + ((size_t)b * Hq + (size_t)grp * kHpHeads * G) * kHeadDim,

@@ -308,11 +308,11 @@ def test_host_step_matches_device_path():
 
 
 # T8: the benchmark configurations at full size, sampled outputs
-@pytest.mark.parametrize("cfg", [2, 3, 4, 5])
-def test_full_size_configs_sampled(cfg):
-    w = wl.CONFIGS[cfg](seed=0)
+@pytest.mark.parametrize("cfg,seed", [(2, 0), (3, 0), (4, 0), (5, 0), (2, 1), (2, 2), (3, 1), (3, 2), (4, 1)])
+def test_full_size_configs_sampled(cfg, seed):
+    w = wl.CONFIGS[cfg](seed=seed)
     dw = run(w)
-    errs = T.compare_sampled(dw, w, seed=cfg, tag=w.name)
+    errs = T.compare_sampled(dw, w, seed=cfg + 10 * seed, tag=w.name)
     print(w.name, errs)
     assert dw.status() == 0
 
