@@ -33,7 +33,7 @@ if str(ROOT) not in sys.path:
 METRIC = "decode-attention KV GB/s and % of B200 HBM peak (Qwen3-4B shape, batched)"
 # dram__bytes_read.sum + dram__bytes_write.sum of one sweep-kernel launch, from the ncu captures summarised in
 # profiles/sweep_kernel_cfg3_ncu.md and profiles/sweep_kernel_cfg4_traffic.md (seed 0)
-NCU_TRAFFIC_BYTES = {3: 2014590000 + 8948224, 4: 4297704192 + 642816}
+NCU_TRAFFIC_BYTES = {3: 2013172000 + 5599744, 4: 4295371264 + 233728}
 FALLBACK_HBM_GBS = 6650.0
 DATASHEET_HBM_GBS = 8000.0
 
