@@ -59,6 +59,11 @@
  * Asynchrony: every call only enqueues work on `cuda_stream` (a cudaStream_t
  * passed as void*, NULL = the legacy default stream) and returns without
  * synchronising, except qf_read_status and qf_decode_step_host, which wait.
+ * qf_decode_partial and qf_combine may be captured into a CUDA graph and
+ * replayed (make one un-captured call per device first: it sets kernel
+ * attributes and builds the TMA descriptors); every replay tags the scratch
+ * words it relies on afresh, so a replay behaves like a new call.  A workspace
+ * serves one call at a time: calls that may overlap on the GPU need their own.
  *
  * Errors: 0 = success.  A negative return means nothing was enqueued.
  * Device-side metadata (table entries, ranges) is not validated unless

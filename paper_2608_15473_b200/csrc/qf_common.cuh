@@ -48,7 +48,8 @@ constexpr int kEpochShift = 10;
 constexpr unsigned long long kEpochLowMask = (1ull << kEpochShift) - 1;
 
 // Header words (unsigned long long) at the start of the workspace.
-enum { kHdrStatus = 0, kHdrLastEpoch = 1, kHdrTotals = 2 /* low: total units, high: units per CTA */ };
+enum { kHdrStatus = 0, kHdrLastEpoch = 1, kHdrTotals = 2 /* low: total units, high: units per CTA */,
+       kHdrLaunchCount = 3 /* bumped by the last CTA of every sweep launch */, kHdrDone = 4 /* epoch-tagged */ };
 
 // OR `bits` into an epoch-tagged word.  Bounded retry; contention is at most a few writers.
 __device__ __forceinline__ void epoch_or(unsigned long long *w, unsigned long long epoch, unsigned bits)
@@ -75,6 +76,21 @@ __device__ __forceinline__ unsigned epoch_arrive(unsigned long long *w, unsigned
         old = prev;
     }
     return 0;
+}
+
+// The epoch of a launch is the host's per-call tag plus a device-side launch count.  The host tag makes
+// every API call distinct; the device count makes every REPLAY of a captured CUDA graph distinct (a
+// replay re-runs the kernel with the captured host tag).  All CTAs read the count at their start; the
+// CTA that finishes last (epoch-tagged done counter) bumps it for the next launch.
+__device__ __forceinline__ unsigned long long launch_epoch(const unsigned long long *header,
+                                                           unsigned long long host_epoch)
+{
+    return (host_epoch + __ldcg(header + kHdrLaunchCount)) & ((1ull << 54) - 1);
+}
+__device__ __forceinline__ void launch_done(unsigned long long *header, unsigned long long epoch, unsigned n_ctas)
+{
+    if (epoch_arrive(header + kHdrDone, epoch) == n_ctas)
+        __stcg(header + kHdrLaunchCount, __ldcg(header + kHdrLaunchCount) + 1);
 }
 
 // Clamp a shard's token range to the request's cached length.

@@ -111,7 +111,7 @@ sweep_hp_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
                 float *__restrict__ o_part, float *__restrict__ m_part, float *__restrict__ lse_part,
                 unsigned long long *__restrict__ header, const int *__restrict__ global_prefix,
                 unsigned long long *__restrict__ counters, float *__restrict__ seg, int seg_stride,
-                unsigned long long epoch, DevParams P)
+                unsigned long long host_epoch, DevParams P)
 {
     extern __shared__ uint8_t smem_raw[];
     HpSmem<G> &sm = *reinterpret_cast<HpSmem<G> *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -132,6 +132,7 @@ sweep_hp_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     }
     grid_dependency_wait();     // nothing above touches global memory
     grid_launch_dependents();
+    const unsigned long long epoch = launch_epoch(header, host_epoch);
     if (blockIdx.x == 0 && tid == 0) header[kHdrLastEpoch] = epoch;
 
     // ---- plan: prefix sum of pages x head groups over (request, shard) entries
@@ -302,7 +303,10 @@ sweep_hp_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
             return;
         }
         const StageMeta mt = sm.meta[stage];
-        if (mt.entry < 0) return;
+        if (mt.entry < 0) {   // end of this CTA's piece
+            if (tid == 0) launch_done(header, epoch, gridDim.x);
+            return;
+        }
 
         if (mt.flags & kSegFirst) {
             const uint16_t *qs = sm.q[stage] + warp * G * kHeadDim;  // this warp's head group rows

@@ -341,3 +341,29 @@ def test_a_wait_that_cannot_be_satisfied_times_out_and_leaves_the_context_usable
     dw.step()
     assert dw.status() == 0
     T.compare_all(dw, w)
+
+
+@pytest.mark.parametrize("flags", [0, qf.QF_FLAG_HEAD_PARALLEL])
+def test_cuda_graph_replay_with_new_queries(flags):
+    # a captured decode step replayed with fresh queries: every replay must behave like a fresh launch
+    # (the scratch words that must "start at zero" are tagged per launch, also under replay)
+    lens = [40_000, 9_000, 123, 17_000]
+    w = wl.make_workload("graph", lens, [wl.fixed_shards(L, 8192) for L in lens], 16, 8, seed=83)
+    dw = DeviceWorkload(w, flags=flags)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        dw.step(s)                      # first call outside capture (one-time set-up), as documented
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            dw.step(s)
+    rng = np.random.default_rng(83)
+    for it in range(3):
+        w.q = wl.f32_to_bf16_bits(rng.standard_normal(w.q.shape).astype(np.float32))
+        dw.q.copy_(torch.from_numpy(w.q.view(np.int16)).view(torch.bfloat16).cuda())
+        dw.poison_outputs()
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        T.compare_all(dw, w, tag=f"replay {it}")
+        assert dw.status() == 0
