@@ -178,8 +178,8 @@ def combine(o_part, lse_part, shard_counts, sh: Shape):
     out = np.zeros((sh.batch, sh.num_q_heads, sh.head_dim), np.float64)
     lse = np.zeros((sh.batch, sh.num_q_heads), np.float64)
     shc = sh.c()
-    rc = lib().qfo_combine(_p(np.ascontiguousarray(o_part), np.float64),
-                           _p(np.ascontiguousarray(lse_part), np.float64),
+    o_part, lse_part = np.ascontiguousarray(o_part), np.ascontiguousarray(lse_part)  # kept alive over the call
+    rc = lib().qfo_combine(_p(o_part, np.float64), _p(lse_part, np.float64),
                            _p(shard_counts, np.int32), ctypes.byref(shc),
                            _p(out, np.float64), _p(lse, np.float64))
     assert rc == 0
@@ -192,8 +192,8 @@ def combine_fold(o_part, lse_part, shard_counts, sh: Shape, perm=None):
     lse = np.zeros((sh.batch, sh.num_q_heads), np.float64)
     pm = None if perm is None else np.ascontiguousarray(np.asarray(perm, np.int32))
     shc = sh.c()
-    rc = lib().qfo_combine_fold(_p(np.ascontiguousarray(o_part), np.float64),
-                                _p(np.ascontiguousarray(lse_part), np.float64),
+    o_part, lse_part = np.ascontiguousarray(o_part), np.ascontiguousarray(lse_part)  # kept alive over the call
+    rc = lib().qfo_combine_fold(_p(o_part, np.float64), _p(lse_part, np.float64),
                                 _p(shard_counts, np.int32), _p(pm, np.int32), ctypes.byref(shc),
                                 _p(out, np.float64), _p(lse, np.float64))
     assert rc == 0
@@ -206,8 +206,8 @@ def self_fold(o_prev, lse_prev, q, k_new, v_new, sh: Shape):
     lse = np.zeros((sh.batch, sh.num_q_heads), np.float64)
     s_self = np.zeros((sh.batch, sh.num_q_heads), np.float64)
     shc = sh.c()
-    rc = lib().qfo_self_fold(_p(np.ascontiguousarray(o_prev), np.float64),
-                             _p(np.ascontiguousarray(lse_prev), np.float64), _p(q, np.uint16),
+    o_prev, lse_prev = np.ascontiguousarray(o_prev), np.ascontiguousarray(lse_prev)  # kept alive over the call
+    rc = lib().qfo_self_fold(_p(o_prev, np.float64), _p(lse_prev, np.float64), _p(q, np.uint16),
                              _p(k_new, np.uint16), _p(v_new, np.uint16), ctypes.byref(shc),
                              _p(out, np.float64), _p(lse, np.float64), _p(s_self, np.float64))
     assert rc == 0

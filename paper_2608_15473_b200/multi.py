@@ -28,3 +28,45 @@ def reduce_timings(times_ms: Dict[str, float], counts: Dict[str, float], dist=No
 def whole_job_throughput(total_bytes: float, max_ms_per_step: float) -> float:
     """GB/s of the whole job: bytes all ranks processed per step over the slowest rank's step time."""
     return total_bytes / (max_ms_per_step * 1e-3) / 1e9
+
+
+# --------------------------------------------------------------------------------------------------
+# One request's cache split over devices (Section 5): every device sweeps the shards it holds and
+# returns (O, log Z) per shard; the owner merges.  The states are tiny (one "j-th" of the sweep's
+# bytes), so the exchange is a gather of [B, S_local, Hq, D] + [B, S_local, Hq] per rank.  On GPUs
+# the same exchange needs no collective at all if o_part / lse_part passed to qf_decode_partial are
+# peer-mapped pointers into the owner's buffers: the sweep kernel writes shard states with plain
+# stores, so its epilogue is the transfer ("parked, not pushed").
+# --------------------------------------------------------------------------------------------------
+def shard_slice(max_shards: int, world_size: int, rank: int) -> range:
+    """Shard slots [lo, hi) of every request that ``rank`` sweeps: equal blocks of ceil(S/world)."""
+    per = -(-max_shards // world_size)
+    lo = min(max_shards, rank * per)
+    return range(lo, min(max_shards, lo + per))
+
+
+def local_shard_ranges(shard_ranges, max_shards: int, world_size: int, rank: int):
+    """The rank's view of the shard table: [B, S_local, 2] with S_local = ceil(S/world), padded with
+    empty ranges (0, 0) so that every rank sweeps the same number of slots."""
+    per = -(-max_shards // world_size)
+    sl = shard_slice(max_shards, world_size, rank)
+    out = torch.zeros((shard_ranges.shape[0], per, 2), dtype=shard_ranges.dtype, device=shard_ranges.device)
+    out[:, :len(sl)] = shard_ranges[:, sl.start:sl.stop]
+    return out
+
+
+def gather_shard_states(o_local: torch.Tensor, lse_local: torch.Tensor, max_shards: int, dist):
+    """All ranks' shard states, concatenated in shard order: o [B, S, Hq, D], lse [B, S, Hq].
+
+    o_local [B, S_local, Hq, D], lse_local [B, S_local, Hq]; padded slots carry lse = -inf and are
+    dropped.  Every rank receives the result (an all-gather keeps the code path identical on gloo and
+    NCCL); only the owner needs it.
+    """
+    world = dist.get_world_size()
+    o_all = [torch.empty_like(o_local) for _ in range(world)]
+    l_all = [torch.empty_like(lse_local) for _ in range(world)]
+    dist.all_gather(o_all, o_local.contiguous())
+    dist.all_gather(l_all, lse_local.contiguous())
+    o = torch.cat(o_all, dim=1)[:, :max_shards]
+    lse = torch.cat(l_all, dim=1)[:, :max_shards]
+    return o, lse

@@ -68,3 +68,48 @@ def test_split_requests_is_a_partition():
 def test_single_process_reduction_is_identity():
     t, c = reduce_timings({"a": 1.5}, {"b": 2.0}, None)
     assert t == {"a": 1.5} and c == {"b": 2.0}
+
+
+# ---- one request's cache split over ranks (Section 5): plumbing of the shard-state exchange
+def _sharded_rank(rank, world, port, out_dir):
+    from oracle import qf_oracle as orc
+    from paper_2608_15473_b200.multi import gather_shard_states, local_shard_ranges, shard_slice
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        lens = [1000, 37, 0, 513]
+        S = 5                                                    # not a multiple of the world size
+        w = wl.make_workload("split", lens, [wl.even_shards(L, S) for L in lens], 4, 2, seed=91)
+        q = torch.from_numpy(w.q.view(np.uint8).copy())         # raw bytes of the bf16 query
+        if rank != 0:
+            q.zero_()
+        dist.broadcast(q, src=0)                                 # only the query travels
+        local = local_shard_ranges(torch.from_numpy(w.shard_ranges), S, world, rank).numpy()
+        sh = orc.Shape(batch=w.batch, num_q_heads=4, num_kv_heads=2, max_pages_per_req=w.max_pages_per_req,
+                       max_shards=local.shape[1])
+        # the device-side sweep of this rank's shards (the CPU oracle stands in for the GPU here)
+        o_loc, _, l_loc = orc.decode_partial(q.numpy().view(np.uint16).reshape(w.q.shape), w.k_cache, w.v_cache, w.block_table,
+                                             w.seq_lens, np.ascontiguousarray(local), sh)
+        o, lse = gather_shard_states(torch.from_numpy(o_loc), torch.from_numpy(l_loc), S, dist)
+        if rank == 0:                                            # the owner merges
+            sh_all = orc.Shape(batch=w.batch, num_q_heads=4, num_kv_heads=2,
+                               max_pages_per_req=w.max_pages_per_req, max_shards=S)
+            out, lse_out = orc.combine(o.numpy(), lse.numpy(), None, sh_all)
+            ref_out, ref_lse = orc.decode_full(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, sh_all)
+            np.save(os.path.join(out_dir, "err.npy"),
+                    np.array([np.abs(out - ref_out).max(),
+                              np.abs(np.where(np.isneginf(ref_lse), 0, lse_out - ref_lse)).max(),
+                              float(np.array_equal(np.isneginf(lse_out), np.isneginf(ref_lse))),
+                              float(list(shard_slice(S, world, 0)) == [0, 1, 2]),
+                              float(list(shard_slice(S, world, 1)) == [3, 4])]))
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_request_split_over_two_ranks_merges_to_the_unsplit_result(tmp_path):
+    world, port = 2, _free_port()
+    mp.spawn(_sharded_rank, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    err = np.load(tmp_path / "err.npy")
+    assert err[0] < 1e-13 and err[1] < 1e-12 and err[2] == 1.0 and err[3] == 1.0 and err[4] == 1.0
