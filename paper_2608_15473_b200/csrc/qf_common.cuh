@@ -87,9 +87,26 @@ __device__ __forceinline__ unsigned long long launch_epoch(const unsigned long l
 {
     return (host_epoch + __ldcg(header + kHdrLaunchCount)) & ((1ull << 54) - 1);
 }
+// Arrival on an epoch-tagged counter that many CTAs hit at the same moment (44-bit tag, 20-bit count).
+// The common case is one atomicAdd (a compare-and-swap loop collapses when 148 CTAs finish together);
+// only the first arrivals of a launch find a stale word and install a fresh one.  Returns the count
+// after this arrival, or 0 if the bounded retry ran out.
+__device__ __forceinline__ unsigned epoch_arrive_crowd(unsigned long long *w, unsigned long long epoch)
+{
+    const unsigned long long tag = epoch & ((1ull << 44) - 1);
+    for (int tries = 0; tries < (1 << 12); ++tries) {
+        const unsigned long long old = atomicAdd(w, 1ull);
+        if ((old >> 20) == tag) return (unsigned)(old & 0xFFFFFull) + 1u;
+        // stale word (and our increment left it stale): try to replace it by "tag, one arrival"
+        const unsigned long long cur = *reinterpret_cast<volatile unsigned long long *>(w);
+        if ((cur >> 20) == tag) continue;   // someone else installed the fresh word: arrive again
+        if (atomicCAS(w, cur, (tag << 20) | 1ull) == cur) return 1u;
+    }
+    return 0u;
+}
 __device__ __forceinline__ void launch_done(unsigned long long *header, unsigned long long epoch, unsigned n_ctas)
 {
-    if (epoch_arrive(header + kHdrDone, epoch) == n_ctas)
+    if (epoch_arrive_crowd(header + kHdrDone, epoch) == n_ctas)
         __stcg(header + kHdrLaunchCount, __ldcg(header + kHdrLaunchCount) + 1);
 }
 
