@@ -35,6 +35,22 @@ struct DevParams {
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Loads of words that other CTAs (or the previous kernel of the stream) have just written: L2-coherent
+// (.cg) and pinned in program order.  The __ldcg intrinsic is a plain asm without a memory clobber, so
+// the compiler may move it above a fence or a grid-dependency wait; these may not be moved.
+__device__ __forceinline__ float ld_sync_f32(const float *p)
+{
+    float v;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned long long ld_sync_u64(const unsigned long long *p)
+{
+    unsigned long long v;
+    asm volatile("ld.global.cg.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000u); }
 
 // bf16 pair packed in a 32-bit word -> two fp32 (exact).
@@ -78,36 +94,44 @@ __device__ __forceinline__ unsigned epoch_arrive(unsigned long long *w, unsigned
     return 0;
 }
 
-// The epoch of a launch is the host's per-call tag plus a device-side launch count.  The host tag makes
-// every API call distinct; the device count makes every REPLAY of a captured CUDA graph distinct (a
-// replay re-runs the kernel with the captured host tag).  All CTAs read the count at their start; the
-// CTA that finishes last (epoch-tagged done counter) bumps it for the next launch.
+// The epoch of a launch pairs the host's per-call tag (upper 30 bits) with a device-side launch count
+// (lower 24 bits).  The host tag makes every API call distinct; the device count makes every REPLAY of
+// a captured CUDA graph distinct (a replay re-runs the kernel with the captured host tag).  The pair is
+// kept as two fields, not a sum, so that an old graph replayed after newer calls cannot land on an
+// epoch a newer call used.  One thread per CTA reads the count at the CTA's start (the caller shares it
+// through shared memory); the CTA that finishes last (epoch-tagged done counter) bumps it for the next launch.
 __device__ __forceinline__ unsigned long long launch_epoch(const unsigned long long *header,
                                                            unsigned long long host_epoch)
 {
-    return (host_epoch + __ldcg(header + kHdrLaunchCount)) & ((1ull << 54) - 1);
+    // an atomic read: performed at the L2 point of coherence, like the bump in launch_done
+    const unsigned long long count = atomicAdd(const_cast<unsigned long long *>(header) + kHdrLaunchCount, 0ull);
+    return ((host_epoch & ((1ull << 30) - 1)) << 24) | (count & ((1ull << 24) - 1));
 }
 // Arrival on an epoch-tagged counter that many CTAs hit at the same moment (44-bit tag, 20-bit count).
-// The common case is one atomicAdd (a compare-and-swap loop collapses when 148 CTAs finish together);
-// only the first arrivals of a launch find a stale word and install a fresh one.  Returns the count
+// The common case is one read and one atomicAdd (a compare-and-swap loop on the count collapses when 148
+// CTAs finish together); only the first arrivals of a launch find a stale word and install a fresh one.  Returns the count
 // after this arrival, or 0 if the bounded retry ran out.
 __device__ __forceinline__ unsigned epoch_arrive_crowd(unsigned long long *w, unsigned long long epoch)
 {
     const unsigned long long tag = epoch & ((1ull << 44) - 1);
     for (int tries = 0; tries < (1 << 12); ++tries) {
-        const unsigned long long old = atomicAdd(w, 1ull);
-        if ((old >> 20) == tag) return (unsigned)(old & 0xFFFFFull) + 1u;
-        // stale word (and our increment left it stale): try to replace it by "tag, one arrival"
         const unsigned long long cur = *reinterpret_cast<volatile unsigned long long *>(w);
-        if ((cur >> 20) == tag) continue;   // someone else installed the fresh word: arrive again
-        if (atomicCAS(w, cur, (tag << 20) | 1ull) == cur) return 1u;
+        if ((cur >> 20) == tag) {
+            // fresh word: one atomicAdd, no retry loop
+            const unsigned long long old = atomicAdd(w, 1ull);
+            if ((old >> 20) == tag) return (unsigned)(old & 0xFFFFFull) + 1u;
+        } else if (atomicCAS(w, cur, (tag << 20) | 1ull) == cur) {
+            // stale word: nobody touches it except through this compare-and-swap, so exactly one
+            // arrival installs the fresh word (and is its first count); the others see it next time round
+            return 1u;
+        }
     }
     return 0u;
 }
 __device__ __forceinline__ void launch_done(unsigned long long *header, unsigned long long epoch, unsigned n_ctas)
 {
     if (epoch_arrive_crowd(header + kHdrDone, epoch) == n_ctas)
-        __stcg(header + kHdrLaunchCount, __ldcg(header + kHdrLaunchCount) + 1);
+        atomicAdd(header + kHdrLaunchCount, 1ull);
 }
 
 // Clamp a shard's token range to the request's cached length.

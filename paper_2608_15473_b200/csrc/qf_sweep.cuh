@@ -145,6 +145,7 @@ struct SweepSmem {
     alignas(8) unsigned long long empty_bar[kStages];
     alignas(8) unsigned long long red_bar[2];
     int abort_flag;
+    unsigned long long epoch;   // this launch's epoch, read once per CTA
     int is_last;
     int scan_ws[kConsumerWarps + 1];
     int prefix[kMaxSmemEntries + 1];
@@ -167,7 +168,7 @@ __device__ __forceinline__ void merge_segments(const float *__restrict__ seg, in
 #pragma unroll
             for (int u = 0; u < kBatch; ++u)
                 mv[u] = (base + u < nseg)
-                            ? __ldcg(seg + (size_t)(first_slot + (base + u) * slot_step) * seg_stride + G * kHeadDim + 2 * head)
+                            ? ld_sync_f32(seg + (size_t)(first_slot + (base + u) * slot_step) * seg_stride + G * kHeadDim + 2 * head)
                             : neg_inf();
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) M = fmaxf(M, mv[u]);
@@ -181,9 +182,9 @@ __device__ __forceinline__ void merge_segments(const float *__restrict__ seg, in
             for (int u = 0; u < kBatch; ++u) {
                 const bool on = base + u < nseg;
                 const float *sl = seg + (size_t)(first_slot + (on ? base + u : 0) * slot_step) * seg_stride;
-                mv[u] = on ? __ldcg(sl + G * kHeadDim + 2 * head) : neg_inf();
-                zv[u] = on ? __ldcg(sl + G * kHeadDim + 2 * head + 1) : 0.f;
-                av[u] = on ? __ldcg(sl + head * kHeadDim + d) : 0.f;
+                mv[u] = on ? ld_sync_f32(sl + G * kHeadDim + 2 * head) : neg_inf();
+                zv[u] = on ? ld_sync_f32(sl + G * kHeadDim + 2 * head + 1) : 0.f;
+                av[u] = on ? ld_sync_f32(sl + head * kHeadDim + d) : 0.f;
             }
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) {   // fixed order: deterministic
@@ -232,8 +233,10 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     }
     grid_dependency_wait();     // nothing above touches global memory
     grid_launch_dependents();
-    const unsigned long long epoch = launch_epoch(header, host_epoch);
-    if (blockIdx.x == 0 && tid == 0) header[kHdrLastEpoch] = epoch;
+    if (tid == 0) {
+        sm.epoch = launch_epoch(header, host_epoch);
+        if (blockIdx.x == 0) header[kHdrLastEpoch] = sm.epoch;
+    }
 
     // ---- plan: prefix sum over (request, shard) entries, in shared memory when it fits
     const int *prefix;
@@ -269,6 +272,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
         __syncthreads();
         prefix = sm.prefix;
     }
+    const unsigned long long epoch = sm.epoch;   // written before the plan's barriers
     const int total = prefix[n_entries];
     const int per_cta = (total + (int)gridDim.x - 1) / (int)gridDim.x;
     const long long pos0_ll = (long long)blockIdx.x * per_cta;

@@ -35,6 +35,7 @@ struct HpSmem {
     alignas(8) unsigned long long full_bar[kHpStages];
     alignas(8) unsigned long long empty_bar[kHpStages];
     int abort_flag;
+    unsigned long long epoch;   // this launch's epoch, read once per CTA
     int scan_ws[kConsumerWarps + 1];
     int prefix[kMaxSmemEntries + 1];
 };
@@ -71,7 +72,7 @@ __device__ __forceinline__ void merge_pieces(const float *__restrict__ seg, int 
             float mv[kBatch];
 #pragma unroll
             for (int u = 0; u < kBatch; ++u)
-                mv[u] = (base + u < nseg) ? __ldcg(slot_of(base + u) + G * kHeadDim + 2 * head) : neg_inf();
+                mv[u] = (base + u < nseg) ? ld_sync_f32(slot_of(base + u) + G * kHeadDim + 2 * head) : neg_inf();
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) M = fmaxf(M, mv[u]);
         }
@@ -84,9 +85,9 @@ __device__ __forceinline__ void merge_pieces(const float *__restrict__ seg, int 
             for (int u = 0; u < kBatch; ++u) {
                 const bool on = base + u < nseg;
                 const float *sl = slot_of(on ? base + u : 0);
-                mv[u] = on ? __ldcg(sl + G * kHeadDim + 2 * head) : neg_inf();
-                zv[u] = on ? __ldcg(sl + G * kHeadDim + 2 * head + 1) : 0.f;
-                av[u] = on ? __ldcg(sl + head * kHeadDim + d) : 0.f;
+                mv[u] = on ? ld_sync_f32(sl + G * kHeadDim + 2 * head) : neg_inf();
+                zv[u] = on ? ld_sync_f32(sl + G * kHeadDim + 2 * head + 1) : 0.f;
+                av[u] = on ? ld_sync_f32(sl + head * kHeadDim + d) : 0.f;
             }
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) {   // fixed order: deterministic
@@ -132,8 +133,10 @@ sweep_hp_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     }
     grid_dependency_wait();     // nothing above touches global memory
     grid_launch_dependents();
-    const unsigned long long epoch = launch_epoch(header, host_epoch);
-    if (blockIdx.x == 0 && tid == 0) header[kHdrLastEpoch] = epoch;
+    if (tid == 0) {
+        sm.epoch = launch_epoch(header, host_epoch);
+        if (blockIdx.x == 0) header[kHdrLastEpoch] = sm.epoch;
+    }
 
     // ---- plan: prefix sum of pages x head groups over (request, shard) entries
     const int *prefix;
@@ -169,6 +172,7 @@ sweep_hp_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         __syncthreads();
         prefix = sm.prefix;
     }
+    const unsigned long long epoch = sm.epoch;   // written before the plan's barriers
     const int total = prefix[n_entries];
     Pieces pc;
     pc.init(total, (int)gridDim.x);
