@@ -131,3 +131,45 @@ def test_append_skips_requests_without_a_page():
     # request 0 is full (position 16 needs a second page that does not exist): untouched; request 1 got its row
     p1 = int(w.block_table[1, 0])
     assert int(diff.sum()) == int(diff[p1, :, 5].sum()) and int(diff[p1, :, 5].sum()) > 0
+
+
+def test_decode_loop_is_a_fold_over_steps():
+    # Twenty decode steps: sweep the cache, fold the current token in, append it, advance.  After every step
+    # the result must equal attention over all positions so far plus the current one (the appendix's fold).
+    lens0 = [0, 14, 250, 1000]
+    steps = 20
+    Hq, Hkv = 16, 8
+    cap = [L + steps for L in lens0]
+    # pages for the final lengths are allocated up front; the sweep only ever sees seq_lens positions
+    w = wl.make_workload("loop", cap, [wl.fixed_shards(c, 512) for c in cap], Hq, Hkv, seed=97)
+    w.seq_lens = np.asarray(lens0, np.int32)
+    rng = np.random.default_rng(97)
+    dw = DeviceWorkload(w)
+    dw.seq_lens.copy_(torch.from_numpy(w.seq_lens).cuda())
+    sh = T.oracle_shape(w)
+    out = torch.empty_like(dw.out)
+    lse = torch.empty_like(dw.lse)
+    for j in range(steps):
+        qj = wl.f32_to_bf16_bits(rng.standard_normal(w.q.shape).astype(np.float32))
+        kj = wl.f32_to_bf16_bits(rng.standard_normal((w.batch, Hkv, 128)).astype(np.float32))
+        vj = wl.f32_to_bf16_bits(rng.standard_normal((w.batch, Hkv, 128)).astype(np.float32))
+        dw.q.copy_(dev_bf16(qj))
+        dk, dv = dev_bf16(kj), dev_bf16(vj)
+        dw.sweep()
+        qf.combine_self(dw.o_part, dw.lse_part, dw.shard_counts, dw.q, dk, dv, out, lse, dw.params)
+        qf.append_kv(dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens, dk, dv, dw.params)
+        dw.seq_lens += 1
+        torch.cuda.synchronize()
+        # host mirror of the cache, then the oracle over the positions including the current one
+        for b in range(w.batch):
+            L = int(w.seq_lens[b])
+            w.k_cache[w.block_table[b, L // 16], :, L % 16] = kj[b]
+            w.v_cache[w.block_table[b, L // 16], :, L % 16] = vj[b]
+        w.seq_lens = w.seq_lens + 1
+        w.q = qj
+        ref_out, ref_lse = orc.decode_full(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, sh)
+        assert T.out_err(out.cpu().numpy(), ref_out) <= T.ENG_OUT, j
+        assert T.lse_err(lse.cpu().numpy(), ref_lse) <= T.ENG_LSE, j
+    # the device cache equals the host mirror bit for bit
+    kc = dw.k_cache.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(kc, w.k_cache)
