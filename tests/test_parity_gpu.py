@@ -367,3 +367,33 @@ def test_cuda_graph_replay_with_new_queries(flags):
         torch.cuda.synchronize()
         T.compare_all(dw, w, tag=f"replay {it}")
         assert dw.status() == 0
+
+
+@pytest.mark.parametrize("seed", list(range(24)))
+def test_randomized_shapes_and_ranges(seed):
+    # random batch, head counts, group size, lengths, unaligned / overlapping / empty shard ranges, pool slack
+    rng = np.random.default_rng(1000 + seed)
+    Hkv = int(rng.choice([1, 2, 3, 4, 8, 16]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    B = int(rng.integers(1, 9))
+    S = int(rng.integers(1, 7))
+    lens = [int(x) for x in rng.choice([0, 1, 15, 16, 17, 127, 128, 129, 500, 3000, 20000], size=B)]
+    ranges = []
+    for L in lens:
+        rr = []
+        for _ in range(S):
+            kind = rng.integers(4)
+            if kind == 0 or L == 0:
+                rr.append((0, 0))
+            elif kind == 1:
+                rr.append((0, L))
+            else:
+                a, b = sorted(int(x) for x in rng.integers(-3, L + 5, size=2))
+                rr.append((a, b))
+        ranges.append(rr)
+    flags = int(rng.choice([0, 0, qf.QF_FLAG_HEAD_PARALLEL, qf.QF_FLAG_CHECK_BOUNDS]))
+    w = wl.make_workload("fuzz", lens, ranges, Hkv * G, Hkv, seed=seed, pool_factor=float(rng.choice([1.0, 1.5])),
+                         poison_unused=True, poison_tails=True, max_pages_per_req=max(1, (max(lens) + 15) // 16 + 2))
+    dw = run(w, flags)
+    T.compare_all(dw, w, tag=f"seed={seed} Hkv={Hkv} G={G} B={B} S={S} flags={flags}")
+    assert dw.status() == 0
