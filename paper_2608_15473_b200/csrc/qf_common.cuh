@@ -51,6 +51,13 @@ __device__ __forceinline__ unsigned long long ld_sync_u64(const unsigned long lo
     return v;
 }
 
+__device__ __forceinline__ int4 ld_sync_int4(const int4 *p)
+{
+    int4 v;
+    asm volatile("ld.global.cg.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000u); }
 
 // bf16 pair packed in a 32-bit word -> two fp32 (exact).
@@ -65,7 +72,8 @@ constexpr unsigned long long kEpochLowMask = (1ull << kEpochShift) - 1;
 
 // Header words (unsigned long long) at the start of the workspace.
 enum { kHdrStatus = 0, kHdrLastEpoch = 1, kHdrTotals = 2 /* low: total units, high: units per CTA */,
-       kHdrLaunchCount = 3 /* bumped by the last CTA of every sweep launch */, kHdrDone = 4 /* epoch-tagged */ };
+       kHdrLaunchCount = 3 /* bumped by the last CTA of every sweep launch */, kHdrDone = 4 /* epoch-tagged */,
+       kHdrChunk = 5 /* epoch-tagged draw counter of the unit kernel's dynamic chunks */ };
 
 // OR `bits` into an epoch-tagged word.  Bounded retry; contention is at most a few writers.
 __device__ __forceinline__ void epoch_or(unsigned long long *w, unsigned long long epoch, unsigned bits)
@@ -127,6 +135,16 @@ __device__ __forceinline__ unsigned epoch_arrive_crowd(unsigned long long *w, un
         }
     }
     return 0u;
+}
+// A counter that is drawn from with a bare atomicAdd (whose result the drawer needs only much later, so
+// the round trip is off its critical path) must carry the launch's tag BEFORE the first draw.  Every CTA
+// calls this once in its prologue; when it returns the word is (tag << 20 | count so far): either this
+// call installed it, or another CTA's did (then the compare-and-swap fails and changes nothing).
+__device__ __forceinline__ void epoch_counter_open(unsigned long long *w, unsigned long long epoch)
+{
+    const unsigned long long tag = epoch & ((1ull << 44) - 1);
+    const unsigned long long cur = atomicAdd(w, 0ull);
+    if ((cur >> 20) != tag) atomicCAS(w, cur, tag << 20);
 }
 __device__ __forceinline__ void launch_done(unsigned long long *header, unsigned long long epoch, unsigned n_ctas)
 {

@@ -46,9 +46,17 @@ constexpr int kMaxSweepCtas  = 160;               // persistent CTAs (one per SM
 constexpr int kHalfTileBytes = 2048;              // 16 rows x 64 channels of bf16
 constexpr int kRedStride     = kHeadDim + 4;      // padded row of the warp-merge buffer
 constexpr int kMaxSmemEntries = 2048;             // (request, shard) pairs planned in shared memory
+// Tail balancing of the unit kernel: the last 1/kDynDivisor of the stage-unit space is cut into chunks that
+// the CTAs draw from a counter as they run out of work (see PieceGrid).
+constexpr int kDynDivisor       = 12;
+constexpr int kDynMinChunk      = 4;              // stage units
+constexpr int kMaxDynChunks     = 592;            // bounds the segment slots; chunks grow beyond kDynMinChunk to fit
+constexpr int kDynMinUnitsPerCta = 64;            // shorter sweeps stay fully static
+static_assert(kMaxSweepCtas + kMaxDynChunks < (1 << kEpochShift), "segments of one unit must fit the arrival count");
 
 struct WorkspaceLayout {
-    size_t header_off, prefix_off, counter_off, seg_off, total;
+    size_t header_off, prefix_off, counter_off, piece_off, seg_off, total;
+    size_t seg_slots;
     int seg_stride;  // floats per segment slot
 };
 
@@ -62,12 +70,14 @@ inline WorkspaceLayout workspace_layout(int batch, int max_shards, int num_kv_he
     L.header_off = 0;
     L.prefix_off = 256;
     L.counter_off = up(L.prefix_off + (entries + 1) * sizeof(int));
-    L.seg_off = up(L.counter_off + entries * num_kv_heads * sizeof(unsigned long long));
+    L.piece_off = up(L.counter_off + entries * num_kv_heads * sizeof(unsigned long long));
+    L.seg_off = up(L.piece_off + (size_t)(kMaxSweepCtas + kMaxDynChunks) * sizeof(int4));
     L.seg_stride = seg_stride_floats(G);
-    // unit kernel: slot = unit + CTA; head-parallel kernel: two slot groups of eight heads per CTA
-    const size_t unit_slots = entries * num_kv_heads + (size_t)kMaxSweepCtas;
+    // unit kernel: slot = unit + piece; head-parallel kernel: two slot groups of eight heads per CTA
+    const size_t unit_slots = entries * num_kv_heads + (size_t)kMaxSweepCtas + (size_t)kMaxDynChunks;
     const size_t hp_slots = (num_kv_heads % 8 == 0 && G <= 4) ? (size_t)kMaxSweepCtas * 2 * 8 : 0;
     const size_t slots = unit_slots > hp_slots ? unit_slots : hp_slots;
+    L.seg_slots = slots;
     L.total = up(L.seg_off + slots * L.seg_stride * sizeof(float));
     return L;
 }
@@ -84,6 +94,50 @@ __device__ __forceinline__ int entry_units(const int *__restrict__ seq_lens, con
     const int npages = ((end - 1) >> 4) - (beg >> 4) + 1;
     if (hp_groups > 0) return npages * hp_groups;
     return ((npages + kPagesPerStage - 1) / kPagesPerStage) * num_kv_heads;
+}
+
+// The stage-unit space [0, total) is cut into pieces, each swept by one CTA front to back.  Pieces
+// 0..n_ctas-1 are equal static slices of [0, static_end): CTA c starts with piece c.  The rest, when the
+// sweep is long enough to pay for it, is cut into n_chunks chunks of `chunk` units that CTAs draw from a
+// counter when they run out of work: SMs do not stream at the same rate (a few percent, stable per SM),
+// and with static slices alone the slowest SM sets the kernel's time.  The grid of pieces depends only
+// on (total, n_ctas), never on who draws what, so a unit's segments and their merge order are fixed.
+struct PieceGrid {
+    int slice;        // units per static slice (>= 1)
+    int static_end;   // units covered by static slices
+    int chunk;        // units per dynamic chunk (>= 1)
+    int n_chunks;
+};
+__device__ __forceinline__ PieceGrid piece_grid(int total, int n_ctas, bool allow_dynamic)
+{
+    PieceGrid g;
+    if (!allow_dynamic || total < n_ctas * kDynMinUnitsPerCta) {
+        g.slice = max(1, (total + n_ctas - 1) / n_ctas);
+        g.static_end = total;
+        g.chunk = 1;
+        g.n_chunks = 0;
+    } else {
+        g.slice = (total - total / kDynDivisor) / n_ctas;
+        g.static_end = g.slice * n_ctas;
+        const int dyn = total - g.static_end;
+        g.chunk = max(kDynMinChunk, (dyn + kMaxDynChunks - 1) / kMaxDynChunks);
+        g.n_chunks = (dyn + g.chunk - 1) / g.chunk;
+    }
+    return g;
+}
+__device__ __forceinline__ int piece_of(const PieceGrid &g, int n_ctas, int pos)
+{
+    return pos < g.static_end ? pos / g.slice : n_ctas + (pos - g.static_end) / g.chunk;
+}
+__device__ __forceinline__ void piece_range(const PieceGrid &g, int n_ctas, int total, int piece, int &pos0, int &pos1)
+{
+    if (piece < n_ctas) {
+        pos0 = (int)min((long long)g.static_end, (long long)piece * g.slice);
+        pos1 = (int)min((long long)g.static_end, (long long)(piece + 1) * g.slice);
+    } else {
+        pos0 = g.static_end + (piece - n_ctas) * g.chunk;
+        pos1 = min(total, pos0 + g.chunk);
+    }
 }
 
 // ------------------------------------------------------------------ plan kernel (large batches only)
@@ -128,7 +182,9 @@ struct __align__(16) StageMeta {
     int tok_beg;   // clamped shard range
     int tok_end;
     int flags;     // bit0 first stage of a segment, bit1 last stage; bits 8..: segments the unit is cut into
-    int aux;       // bits 0..7: pages whose table entry was out of range; bits 8..: first segment slot of the unit
+    int aux;       // bits 0..7: pages whose table entry was out of range
+    int slot;      // this segment's slot: the unit's first slot + the segment's ordinal (used when the unit is cut)
+    int pad[3];
 };
 enum { kSegFirst = 1, kSegLast = 2 };
 
@@ -146,13 +202,15 @@ struct SweepSmem {
     alignas(8) unsigned long long red_bar[2];
     int abort_flag;
     unsigned long long epoch;   // this launch's epoch, read once per CTA
-    int is_last;
     int scan_ws[kConsumerWarps + 1];
     int prefix[kMaxSmemEntries + 1];
 };
 
 // Merge segments [first, first+nseg) of one (shard, KV head) unit into its final state.
 // Called by the NT threads (a warp or all consumer warps) that arrived last; fixed order, so deterministic.
+// A thread owns outputs idx = tid + k*NT and handles two of them at a time; per pair it walks the segments
+// in batches of eight with all of a batch's loads in flight together (one L2 round trip per batch) and a
+// running maximum, so a unit cut into up to eight segments costs one round trip per output pair.
 template <int G, int NT>
 __device__ __forceinline__ void merge_segments(const float *__restrict__ seg, int seg_stride, int first_slot,
                                                int slot_step, int nseg, size_t out_row, float *__restrict__ o_part,
@@ -160,43 +218,59 @@ __device__ __forceinline__ void merge_segments(const float *__restrict__ seg, in
 {
     const float kLn2 = 0.6931471805599453f;
     constexpr int kBatch = 8;   // segments whose loads are in flight together
-    for (int idx = tid; idx < G * kHeadDim; idx += NT) {
-        const int head = idx >> 7, d = idx & 127;
-        float M = neg_inf();
-        for (int base = 0; base < nseg; base += kBatch) {
-            float mv[kBatch];
+    constexpr int kPair = 2;    // outputs a thread merges together
+    for (int idx0 = tid; idx0 < G * kHeadDim; idx0 += kPair * NT) {
+        float M[kPair], z[kPair], acc[kPair];
+        int head[kPair], d[kPair];
+        bool on_o[kPair];
 #pragma unroll
-            for (int u = 0; u < kBatch; ++u)
-                mv[u] = (base + u < nseg)
-                            ? ld_sync_f32(seg + (size_t)(first_slot + (base + u) * slot_step) * seg_stride + G * kHeadDim + 2 * head)
-                            : neg_inf();
-#pragma unroll
-            for (int u = 0; u < kBatch; ++u) M = fmaxf(M, mv[u]);
+        for (int o = 0; o < kPair; ++o) {
+            const int idx = idx0 + o * NT;
+            on_o[o] = idx < G * kHeadDim;
+            head[o] = on_o[o] ? idx >> 7 : 0;
+            d[o] = idx & 127;
+            M[o] = neg_inf(); z[o] = 0.f; acc[o] = 0.f;
         }
-        const bool empty = (M == neg_inf());
-        const float Ms = empty ? 0.f : M;
-        float z = 0.f, wsum = 0.f;
         for (int base = 0; base < nseg; base += kBatch) {
-            float mv[kBatch], zv[kBatch], av[kBatch];
+            float mv[kPair][kBatch], zv[kPair][kBatch], av[kPair][kBatch];
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) {
                 const bool on = base + u < nseg;
                 const float *sl = seg + (size_t)(first_slot + (on ? base + u : 0) * slot_step) * seg_stride;
-                mv[u] = on ? ld_sync_f32(sl + G * kHeadDim + 2 * head) : neg_inf();
-                zv[u] = on ? ld_sync_f32(sl + G * kHeadDim + 2 * head + 1) : 0.f;
-                av[u] = on ? ld_sync_f32(sl + head * kHeadDim + d) : 0.f;
+#pragma unroll
+                for (int o = 0; o < kPair; ++o) {
+                    mv[o][u] = on ? ld_sync_f32(sl + G * kHeadDim + 2 * head[o]) : neg_inf();
+                    zv[o][u] = on ? ld_sync_f32(sl + G * kHeadDim + 2 * head[o] + 1) : 0.f;
+                    av[o][u] = on ? ld_sync_f32(sl + head[o] * kHeadDim + d[o]) : 0.f;
+                }
             }
 #pragma unroll
-            for (int u = 0; u < kBatch; ++u) {   // fixed order: deterministic
-                const float ew = fast_exp2(mv[u] - Ms);
-                z = fmaf(zv[u], ew, z);
-                wsum = fmaf(av[u], ew, wsum);
+            for (int o = 0; o < kPair; ++o) {
+                float Mn = M[o];
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) Mn = fmaxf(Mn, mv[o][u]);
+                const float Ms = (Mn == neg_inf()) ? 0.f : Mn;
+                const float keep = fast_exp2(M[o] - Ms);   // 0 while nothing has been merged yet
+                z[o] *= keep;
+                acc[o] *= keep;
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {   // fixed order: deterministic
+                    const float ew = fast_exp2(mv[o][u] - Ms);
+                    z[o] = fmaf(zv[o][u], ew, z[o]);
+                    acc[o] = fmaf(av[o][u], ew, acc[o]);
+                }
+                M[o] = Mn;
             }
         }
-        o_part[(out_row + head) * kHeadDim + d] = empty ? 0.f : wsum / z;
-        if (d == 0) {
-            m_part[out_row + head] = empty ? neg_inf() : M * kLn2;
-            lse_part[out_row + head] = empty ? neg_inf() : (M + log2f(z)) * kLn2;
+#pragma unroll
+        for (int o = 0; o < kPair; ++o) {
+            if (!on_o[o]) continue;
+            const bool empty = (M[o] == neg_inf());
+            o_part[(out_row + head[o]) * kHeadDim + d[o]] = empty ? 0.f : acc[o] / z[o];
+            if (d[o] == 0) {
+                m_part[out_row + head[o]] = empty ? neg_inf() : M[o] * kLn2;
+                lse_part[out_row + head[o]] = empty ? neg_inf() : (M[o] + log2f(z[o])) * kLn2;
+            }
         }
     }
 }
@@ -208,7 +282,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
              const int *__restrict__ seq_lens, const int *__restrict__ shard_ranges,
              float *__restrict__ o_part, float *__restrict__ m_part, float *__restrict__ lse_part,
              unsigned long long *__restrict__ header, const int *__restrict__ global_prefix,
-             unsigned long long *__restrict__ counters, float *__restrict__ seg, int seg_stride,
+             int4 *__restrict__ piece_info, float *__restrict__ seg, int seg_stride,
              unsigned long long host_epoch, DevParams P)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -228,14 +302,17 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
         mbar_init(smem_u32(&sm.red_bar[0]), kConsumerWarps);
         mbar_init(smem_u32(&sm.red_bar[1]), kConsumerWarps);
         sm.abort_flag = 0;
-        sm.is_last = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     grid_dependency_wait();     // nothing above touches global memory
     grid_launch_dependents();
-    if (tid == 0) {
-        sm.epoch = launch_epoch(header, host_epoch);
-        if (blockIdx.x == 0) header[kHdrLastEpoch] = sm.epoch;
+    if (tid == kConsumerThreads) {
+        // the producer warp's first lane is idle during the plan below: it fetches the launch's epoch and
+        // makes sure the chunk counter carries it before anybody draws from it
+        const unsigned long long ep = launch_epoch(header, host_epoch);
+        sm.epoch = ep;
+        if (blockIdx.x == 0) header[kHdrLastEpoch] = ep;
+        epoch_counter_open(header + kHdrChunk, ep);
     }
 
     // ---- plan: prefix sum over (request, shard) entries, in shared memory when it fits
@@ -274,12 +351,11 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     }
     const unsigned long long epoch = sm.epoch;   // written before the plan's barriers
     const int total = prefix[n_entries];
-    const int per_cta = (total + (int)gridDim.x - 1) / (int)gridDim.x;
-    const long long pos0_ll = (long long)blockIdx.x * per_cta;
-    const int pos0 = (int)min((long long)total, pos0_ll);
-    const int pos1 = (int)min((long long)total, pos0_ll + per_cta);
+    const int n_ctas = (int)gridDim.x;
+    // a prefix left in global memory (very large batches) makes locating a piece's first entry slow: static only
+    const PieceGrid pg = piece_grid(total, n_ctas, global_prefix == nullptr);
     if (blockIdx.x == 0 && tid == 0)
-        header[kHdrTotals] = (unsigned long long)(unsigned)total | ((unsigned long long)(unsigned)per_cta << 32);
+        header[kHdrTotals] = (unsigned long long)(unsigned)total | ((unsigned long long)(unsigned)(n_ctas + pg.n_chunks) << 32);
 
     if (warp == kConsumerWarps) {
         // ============================ producer warp ============================
@@ -288,16 +364,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
         uint32_t phase = 0;
         int issued = 0;
         bool ok = true;
-        int pos = pos0;
+        int piece = (int)blockIdx.x;
         int e = 0;
-        if (pos < pos1) {  // largest e with prefix[e] <= pos
-            int lo = 0, hi = n_entries;
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (prefix[mid] <= pos) lo = mid; else hi = mid;
-            }
-            e = lo;
-        }
         // Per-segment metadata is kept off the critical path: a shard's token range and the first batch
         // of its block-table row are the same for all KV heads of the shard, so they are cached in
         // registers; the next non-empty shard's are fetched one segment ahead.
@@ -310,6 +378,25 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             const int lp = min(page0_ + lane, last_page_);
             return block_table ? block_table[rb + lp] : (int)(rb + lp);
         };
+        for (;;) {   // pieces: the static slice, then chunks drawn from the counter
+        int pos, pos1;
+        piece_range(pg, n_ctas, total, piece, pos, pos1);
+        // the next chunk is drawn two stages before this piece's last issue: late enough that a slow SM
+        // does not sit on a reserved chunk, early enough that the counter's latency is hidden
+        const int draw_at = max(pos, pos1 - 2);
+        unsigned long long drawn = 0;
+        if (pg.n_chunks > 0 && pos >= pos1 && lane == 0) drawn = atomicAdd(header + kHdrChunk, 1ull);
+        // Every piece leaves one record for the finish kernel: the unit it must merge, if any (see below).
+        const int piece_pos0 = pos;
+        if (pos >= pos1 && lane == 0) piece_info[piece] = make_int4(-1, 0, 0, (int)(unsigned)epoch);
+        if (pos < pos1) {  // largest e with prefix[e] <= pos (pieces are drawn in increasing order)
+            int lo = e, hi = n_entries;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (prefix[mid] <= pos) lo = mid; else hi = mid;
+            }
+            e = lo;
+        }
         while (ok && pos < pos1) {
             while (prefix[e + 1] <= pos) ++e;  // skip empty entries
             const int base = prefix[e];
@@ -335,11 +422,18 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                 }
             }
             const int first_page = beg >> 4, last_page = (end - 1) >> 4;
-            // the CTAs whose slices touch this unit: one segment each
+            // the pieces that touch this unit: one segment each, slot = unit + piece (both increase along
+            // the unit space, so no two segments share a slot)
             const int p0 = base + c * nunits;
-            const int first_cta = p0 / per_cta, last_cta = (p0 + nunits - 1) / per_cta;
-            const int nseg = last_cta - first_cta + 1;
-            const int first_slot = e * Hkv + c + first_cta;
+            const int first_piece = piece_of(pg, n_ctas, p0), last_piece = piece_of(pg, n_ctas, p0 + nunits - 1);
+            const int nseg = last_piece - first_piece + 1;
+            const int first_slot = e * Hkv + c + first_piece;
+            if (pos == piece_pos0 && lane == 0) {
+                // A unit cut into segments is merged by the finish kernel's CTA of the unit's SECOND piece:
+                // that is this piece if it starts inside the unit and the piece before it holds the unit's start.
+                const bool second = (j > 0) && (first_piece == piece - 1);
+                piece_info[piece] = make_int4(second ? e * Hkv + c : -1, first_slot, nseg, (int)(unsigned)epoch);
+            }
 
             // table entries are fetched 32 pages at a time
             int tbl_page0 = 0, tbl = 0;
@@ -370,6 +464,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                 const unsigned bad_mask = __ballot_sync(0xffffffffu, bad && i < np && part == 0) & 0xffu;
                 const bool issuer = (i < np) && (part < 2);
 
+                if (pg.n_chunks > 0 && pos + u == draw_at && lane == 0) drawn = atomicAdd(header + kHdrChunk, 1ull);
                 if (!mbar_wait(smem_u32(&sm.empty_bar[stage]), phase ^ 1, abort_flag)) { ok = false; break; }
                 const bool first = (u == 0), last = (u == seg_len - 1);
                 const uint32_t full = smem_u32(&sm.full_bar[stage]);
@@ -378,7 +473,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                     mt.entry = e; mt.kv_head = c; mt.page0 = page0; mt.npages = np;
                     mt.tok_beg = beg; mt.tok_end = end;
                     mt.flags = (first ? kSegFirst : 0) | (last ? kSegLast : 0) | (nseg << 8);
-                    mt.aux = (int)bad_mask | (first_slot << 8);
+                    mt.aux = (int)bad_mask;
+                    mt.slot = e * Hkv + c + piece;
                     sm.meta[stage] = mt;
                     mbar_arrive_expect_tx(full, (uint32_t)np * 2u * kPageBytes + (first ? (uint32_t)G * 256u : 0u));
                     if (bad_mask) epoch_or(header + kHdrStatus, epoch, kStatusBadPage);
@@ -395,6 +491,13 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                 if (++stage == kStages) { stage = 0; phase ^= 1; }
             }
             pos += seg_len;
+        }
+        if (!ok || pg.n_chunks == 0) break;
+        drawn = __shfl_sync(0xffffffffu, drawn, 0);
+        if ((drawn >> 20) != (epoch & ((1ull << 44) - 1))) { ok = false; break; }   // not this launch's counter
+        const int ticket = (int)(drawn & 0xFFFFFull);
+        if (ticket >= pg.n_chunks) break;
+        piece = n_ctas + ticket;
         }
         if (ok) {  // end-of-work marker
             if (mbar_wait(smem_u32(&sm.empty_bar[stage]), phase ^ 1, abort_flag)) {
@@ -462,7 +565,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             return;
         }
         const StageMeta mt = sm.meta[stage];
-        if (mt.entry < 0) {   // end of this CTA's slice
+        if (mt.entry < 0) {   // end of this CTA's work
             if (tid == 0) launch_done(header, epoch, gridDim.x);
             return;
         }
@@ -503,11 +606,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             }
             constexpr int RG = SweepSmem<G>::kRoundHeads;
             const int nseg = mt.flags >> 8;
-            const int first_slot = mt.aux >> 8;
-            const int unit = mt.entry * Hkv + mt.kv_head;
             const size_t out_row = ((size_t)mt.entry * Hq + (size_t)mt.kv_head * G);  // + head
-            // this CTA's segment is the (blockIdx.x - first_cta)-th of the unit; first_slot = unit + first_cta
-            float *seg_slot = seg + (size_t)(unit + (int)blockIdx.x) * seg_stride;
+            float *seg_slot = seg + (size_t)mt.slot * seg_stride;
 #pragma unroll
             for (int hr = 0; hr < G / RG; ++hr) {
 #pragma unroll
@@ -558,27 +658,40 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                         }
                     }
                 }
-                if (nseg > 1) __threadfence();   // segment state visible device-wide before the arrival below
-                if (!red_sync(1, red_phase1)) return;
-            }
-            if (nseg > 1) {
-                // the unit was cut by slice boundaries: whoever arrives last merges all its segments
-                if (tid == 0) {
-                    const unsigned n = epoch_arrive(counters + unit, epoch);
-                    if (n == 0) epoch_or(header + kHdrStatus, epoch, kStatusTimeout);
-                    sm.is_last = (n == (unsigned)nseg) ? 1 : 0;
-                }
-                if (!red_sync(0, red_phase0)) return;
-                const int is_last = *reinterpret_cast<volatile int *>(&sm.is_last);
-                if (is_last) {
-                    __threadfence();
-                    merge_segments<G, kConsumerThreads>(seg, seg_stride, first_slot, 1, nseg, out_row, o_part, m_part, lse_part, tid);
-                }
                 if (!red_sync(1, red_phase1)) return;
             }
         }
         if (++stage == kStages) { stage = 0; phase ^= 1; }
     }
+}
+
+// ------------------------------------------------------------------ finish kernel
+// Merges the units that piece boundaries cut into segments.  CTA p looks at the record piece p left: if
+// the piece is the second one of a cut unit, the CTA merges that unit's segment slots, in slot order,
+// into the unit's final state.  Running after the sweep (not inside it, by whoever arrives last at a
+// counter) keeps the sweep's consumer warps streaming: a merge is a round trip to L2, several
+// microseconds while the memory system is saturated, and it would land on the CTAs that are already
+// late.  A record is used only if it carries this launch's epoch and its numbers fit the workspace, so
+// an aborted sweep cannot make this kernel touch memory outside it.
+template <int G>
+__global__ void __launch_bounds__(kConsumerThreads)
+finish_kernel(const int4 *__restrict__ piece_info, const unsigned long long *__restrict__ header,
+              const float *__restrict__ seg, int seg_stride, int seg_slots, float *__restrict__ o_part,
+              float *__restrict__ m_part, float *__restrict__ lse_part, int n_units, int Hkv, int Hq)
+{
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const int p = (int)blockIdx.x + 1;      // piece 0 is never a second piece
+    const int n_pieces = (int)(ld_sync_u64(header + kHdrTotals) >> 32);
+    if (p >= n_pieces) return;
+    const int4 rec = ld_sync_int4(piece_info + p);
+    const unsigned long long epoch = ld_sync_u64(header + kHdrLastEpoch);
+    if (rec.x < 0 || rec.w != (int)(unsigned)epoch) return;
+    const int unit = rec.x, first_slot = rec.y, nseg = rec.z;
+    if (unit >= n_units || nseg < 2 || first_slot < 0 || (long long)first_slot + nseg > (long long)seg_slots) return;
+    const size_t out_row = (size_t)(unit / Hkv) * Hq + (size_t)(unit % Hkv) * G;
+    merge_segments<G, kConsumerThreads>(seg, seg_stride, first_slot, 1, nseg, out_row, o_part, m_part, lse_part,
+                                        (int)threadIdx.x);
 }
 
 // ------------------------------------------------------------------ bounded-wait self-test
@@ -671,7 +784,7 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
 {
     unsigned long long *header = reinterpret_cast<unsigned long long *>(ws + wsl.header_off);
     int *prefix = reinterpret_cast<int *>(ws + wsl.prefix_off);
-    unsigned long long *counters = reinterpret_cast<unsigned long long *>(ws + wsl.counter_off);
+    int4 *piece_info = reinterpret_cast<int4 *>(ws + wsl.piece_off);
     float *seg = reinterpret_cast<float *>(ws + wsl.seg_off);
     const int n_entries = P.batch * P.max_shards;
     const size_t smem = sizeof(SweepSmem<G>) + 1024;
@@ -694,10 +807,16 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
     }
     if (ev0) cudaEventRecord(ev0, st);
     cudaError_t e = launch_pdl(sweep_kernel<G>, dim3(n_ctas), dim3(kSweepThreads), smem, st, kmap, vmap,
-                               (const uint16_t *)q, bt, sl, sr, o, m, l, header, global_prefix, counters, seg,
+                               (const uint16_t *)q, bt, sl, sr, o, m, l, header, global_prefix, piece_info, seg,
                                wsl.seg_stride, epoch, P);
     if (ev1) cudaEventRecord(ev1, st);
     if (e != cudaSuccess) { snprintf(msg, msg_len, "sweep_kernel launch: %s", cudaGetErrorString(e)); return -5; }
+    *launches += 1;
+    // one CTA per piece that can be a unit's second piece
+    e = launch_pdl(finish_kernel<G>, dim3(n_ctas + kMaxDynChunks - 1), dim3(kConsumerThreads), 0, st,
+                   (const int4 *)piece_info, (const unsigned long long *)header, (const float *)seg, wsl.seg_stride,
+                   (int)wsl.seg_slots, o, m, l, n_entries * P.num_kv_heads, P.num_kv_heads, P.num_q_heads);
+    if (e != cudaSuccess) { snprintf(msg, msg_len, "finish_kernel launch: %s", cudaGetErrorString(e)); return -5; }
     *launches += 1;
     return 0;
 }
