@@ -97,10 +97,15 @@ enum {
 enum {
     QF_FLAG_CHECK_BOUNDS  = 1, /* range-check page indices on the device           */
     QF_FLAG_SIMPLE_KERNEL = 2, /* use the plain-load sweep kernel (validation aid) */
-    QF_FLAG_HEAD_PARALLEL = 4  /* use the head-parallel sweep kernel (needs Hkv a multiple
+    QF_FLAG_HEAD_PARALLEL = 4, /* use the head-parallel sweep kernel (needs Hkv a multiple
                                   of 8 and G <= 4, else ignored): one page of eight KV
                                   heads per ring stage, no cross-warp merges; faster when
                                   shards are short (a few hundred tokens to ~2,000)      */
+    QF_FLAG_DRAW_ALWAYS   = 8  /* default sweep kernel only: hand out the tail of the work
+                                  as drawn chunks however short the sweep is (by default
+                                  only sweeps long enough to gain from it do).  Same
+                                  results up to fp32 summation order; lets small tests
+                                  reach the drawn-chunk path                             */
 };
 
 /* qf_read_status bits */

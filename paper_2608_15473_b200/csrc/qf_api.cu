@@ -52,6 +52,7 @@ qf::DevParams dev_params(const qf_params *p)
     d.max_pages_per_req = p->max_pages_per_req;
     d.max_shards = p->max_shards;
     d.check_bounds = (p->flags & QF_FLAG_CHECK_BOUNDS) ? 1 : 0;
+    d.draw_always = (p->flags & QF_FLAG_DRAW_ALWAYS) ? 1 : 0;
     d.num_pages = p->num_pages;
     d.sm_scale = p->sm_scale > 0.f ? p->sm_scale : 1.0f / std::sqrt((float)p->head_dim);
     return d;

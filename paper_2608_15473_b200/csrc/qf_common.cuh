@@ -24,6 +24,7 @@ struct DevParams {
     int max_pages_per_req;
     int max_shards;
     int check_bounds;
+    int draw_always;         // cut the tail into drawn chunks however short the sweep is
     long long num_pages;
     float sm_scale;
 };

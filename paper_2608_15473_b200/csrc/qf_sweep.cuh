@@ -48,10 +48,20 @@ constexpr int kRedStride     = kHeadDim + 4;      // padded row of the warp-merg
 constexpr int kMaxSmemEntries = 2048;             // (request, shard) pairs planned in shared memory
 // Tail balancing of the unit kernel: the last 1/kDynDivisor of the stage-unit space is cut into chunks that
 // the CTAs draw from a counter as they run out of work (see PieceGrid).
-constexpr int kDynDivisor       = 12;
-constexpr int kDynMinChunk      = 4;              // stage units
-constexpr int kMaxDynChunks     = 592;            // bounds the segment slots; chunks grow beyond kDynMinChunk to fit
-constexpr int kDynMinUnitsPerCta = 64;            // shorter sweeps stay fully static
+#ifndef QF_DYN_DIVISOR
+#define QF_DYN_DIVISOR 10
+#endif
+#ifndef QF_DYN_MIN_CHUNK
+#define QF_DYN_MIN_CHUNK 3
+#endif
+constexpr int kDynDivisor       = QF_DYN_DIVISOR;
+constexpr int kDynMinChunk      = QF_DYN_MIN_CHUNK;   // stage units
+#ifndef QF_DYN_ROUNDS
+#define QF_DYN_ROUNDS 3
+#endif
+constexpr int kDynRounds        = QF_DYN_ROUNDS;      // chunk sizes halve from round to round
+constexpr int kMaxDynChunks     = kDynRounds * kMaxSweepCtas;   // bounds the segment slots
+constexpr int kDynMinUnitsPerCta = 64;                // shorter sweeps stay fully static
 static_assert(kMaxSweepCtas + kMaxDynChunks < (1 << kEpochShift), "segments of one unit must fit the arrival count");
 
 struct WorkspaceLayout {
@@ -98,46 +108,73 @@ __device__ __forceinline__ int entry_units(const int *__restrict__ seq_lens, con
 
 // The stage-unit space [0, total) is cut into pieces, each swept by one CTA front to back.  Pieces
 // 0..n_ctas-1 are equal static slices of [0, static_end): CTA c starts with piece c.  The rest, when the
-// sweep is long enough to pay for it, is cut into n_chunks chunks of `chunk` units that CTAs draw from a
-// counter when they run out of work: SMs do not stream at the same rate (a few percent, stable per SM),
-// and with static slices alone the slowest SM sets the kernel's time.  The grid of pieces depends only
-// on (total, n_ctas), never on who draws what, so a unit's segments and their merge order are fixed.
+// sweep is long enough to pay for it, is cut into chunks that CTAs draw from a counter when they run out
+// of work: SMs do not stream at the same rate (a few percent, stable per SM), and with static slices alone
+// the slowest SM sets the kernel's time.  Chunks come in kDynRounds rounds of at most n_ctas chunks; every
+// round but the last takes half of what is left, so chunk sizes halve and a chunk is never more than a
+// 1/n_ctas share of the work still to be drawn when it is drawn; the kernel's end is then uneven by about
+// one chunk of the last round.  The grid of pieces depends only on (total, n_ctas), never on who draws
+// what, so a unit's segments and their merge order are fixed.
 struct PieceGrid {
     int slice;        // units per static slice (>= 1)
     int static_end;   // units covered by static slices
-    int chunk;        // units per dynamic chunk (>= 1)
     int n_chunks;
+    int r_start[kDynRounds + 1];   // first unit of round r (r_start[kDynRounds] = total)
+    int r_first[kDynRounds + 1];   // first chunk of round r
+    int r_size[kDynRounds];        // units per chunk in round r (the round's last chunk may be shorter)
 };
-__device__ __forceinline__ PieceGrid piece_grid(int total, int n_ctas, bool allow_dynamic)
+__device__ __forceinline__ PieceGrid piece_grid(int total, int n_ctas, bool allow_dynamic, bool always)
 {
     PieceGrid g;
-    if (!allow_dynamic || total < n_ctas * kDynMinUnitsPerCta) {
+    const int min_total = always ? 2 * n_ctas : n_ctas * kDynMinUnitsPerCta;   // static slices of at least one unit
+    if (!allow_dynamic || total < min_total) {
         g.slice = max(1, (total + n_ctas - 1) / n_ctas);
         g.static_end = total;
-        g.chunk = 1;
-        g.n_chunks = 0;
     } else {
         g.slice = (total - total / kDynDivisor) / n_ctas;
         g.static_end = g.slice * n_ctas;
-        const int dyn = total - g.static_end;
-        g.chunk = max(kDynMinChunk, (dyn + kMaxDynChunks - 1) / kMaxDynChunks);
-        g.n_chunks = (dyn + g.chunk - 1) / g.chunk;
     }
+    int off = g.static_end, idx = 0;
+#pragma unroll
+    for (int r = 0; r < kDynRounds; ++r) {
+        const int rem = total - off;
+        const int share = (r == kDynRounds - 1) ? rem : (rem + 1) / 2;
+        const int size = max(kDynMinChunk, (share + n_ctas - 1) / n_ctas);
+        g.r_start[r] = off;
+        g.r_first[r] = idx;
+        g.r_size[r] = size;
+        off += share;
+        idx += (share + size - 1) / size;
+    }
+    g.r_start[kDynRounds] = total;
+    g.r_first[kDynRounds] = idx;
+    g.n_chunks = idx;
     return g;
 }
 __device__ __forceinline__ int piece_of(const PieceGrid &g, int n_ctas, int pos)
 {
-    return pos < g.static_end ? pos / g.slice : n_ctas + (pos - g.static_end) / g.chunk;
+    if (pos < g.static_end) return pos / g.slice;
+    int piece = 0;
+#pragma unroll
+    for (int r = 0; r < kDynRounds; ++r)
+        if (pos >= g.r_start[r] && pos < g.r_start[r + 1]) piece = n_ctas + g.r_first[r] + (pos - g.r_start[r]) / g.r_size[r];
+    return piece;
 }
-__device__ __forceinline__ void piece_range(const PieceGrid &g, int n_ctas, int total, int piece, int &pos0, int &pos1)
+__device__ __forceinline__ void piece_range(const PieceGrid &g, int n_ctas, int piece, int &pos0, int &pos1)
 {
     if (piece < n_ctas) {
         pos0 = (int)min((long long)g.static_end, (long long)piece * g.slice);
         pos1 = (int)min((long long)g.static_end, (long long)(piece + 1) * g.slice);
-    } else {
-        pos0 = g.static_end + (piece - n_ctas) * g.chunk;
-        pos1 = min(total, pos0 + g.chunk);
+        return;
     }
+    const int k = piece - n_ctas;
+    pos0 = pos1 = g.r_start[kDynRounds];
+#pragma unroll
+    for (int r = 0; r < kDynRounds; ++r)
+        if (k >= g.r_first[r] && k < g.r_first[r + 1]) {
+            pos0 = g.r_start[r] + (k - g.r_first[r]) * g.r_size[r];
+            pos1 = min(pos0 + g.r_size[r], g.r_start[r + 1]);
+        }
 }
 
 // ------------------------------------------------------------------ plan kernel (large batches only)
@@ -353,7 +390,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     const int total = prefix[n_entries];
     const int n_ctas = (int)gridDim.x;
     // a prefix left in global memory (very large batches) makes locating a piece's first entry slow: static only
-    const PieceGrid pg = piece_grid(total, n_ctas, global_prefix == nullptr);
+    const PieceGrid pg = piece_grid(total, n_ctas, global_prefix == nullptr, P.draw_always != 0);
     if (blockIdx.x == 0 && tid == 0)
         header[kHdrTotals] = (unsigned long long)(unsigned)total | ((unsigned long long)(unsigned)(n_ctas + pg.n_chunks) << 32);
 
@@ -380,7 +417,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
         };
         for (;;) {   // pieces: the static slice, then chunks drawn from the counter
         int pos, pos1;
-        piece_range(pg, n_ctas, total, piece, pos, pos1);
+        piece_range(pg, n_ctas, piece, pos, pos1);
         // the next chunk is drawn two stages before this piece's last issue: late enough that a slow SM
         // does not sit on a reserved chunk, early enough that the counter's latency is hidden
         const int draw_at = max(pos, pos1 - 2);
@@ -428,12 +465,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             const int first_piece = piece_of(pg, n_ctas, p0), last_piece = piece_of(pg, n_ctas, p0 + nunits - 1);
             const int nseg = last_piece - first_piece + 1;
             const int first_slot = e * Hkv + c + first_piece;
-            if (pos == piece_pos0 && lane == 0) {
-                // A unit cut into segments is merged by the finish kernel's CTA of the unit's SECOND piece:
-                // that is this piece if it starts inside the unit and the piece before it holds the unit's start.
-                const bool second = (j > 0) && (first_piece == piece - 1);
-                piece_info[piece] = make_int4(second ? e * Hkv + c : -1, first_slot, nseg, (int)(unsigned)epoch);
-            }
+            if (pos == piece_pos0 && lane == 0)   // does this piece start inside a unit?  (the finish kernel's input)
+                piece_info[piece] = make_int4(j > 0 ? e * Hkv + c : -1, first_slot, nseg, (int)(unsigned)epoch);
 
             // table entries are fetched 32 pages at a time
             int tbl_page0 = 0, tbl = 0;
@@ -666,32 +699,125 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
 }
 
 // ------------------------------------------------------------------ finish kernel
-// Merges the units that piece boundaries cut into segments.  CTA p looks at the record piece p left: if
-// the piece is the second one of a cut unit, the CTA merges that unit's segment slots, in slot order,
-// into the unit's final state.  Running after the sweep (not inside it, by whoever arrives last at a
-// counter) keeps the sweep's consumer warps streaming: a merge is a round trip to L2, several
-// microseconds while the memory system is saturated, and it would land on the CTAs that are already
-// late.  A record is used only if it carries this launch's epoch and its numbers fit the workspace, so
-// an aborted sweep cannot make this kernel touch memory outside it.
+// Merges the units that piece boundaries cut into segments, after the sweep (not inside it, by whoever
+// arrives last at a counter: a merge is a few round trips to L2, several microseconds each while the
+// memory system is saturated, and it would land on the CTAs that are already late).
+//
+// CTA p looks at the record piece p left.  If the piece starts inside a unit, its segment is the k-th of
+// that unit (k >= 1).  Segments are merged in groups of kFinGroup: the CTAs with k == 1 or k a multiple of
+// kFinGroup lead a group, the others exit.  A unit of one group is finished by its leader.  Otherwise each
+// leader writes its group's partial state over the group's first slot and arrives at the unit's counter;
+// the leader that arrives last merges the partials.  Nobody waits for anybody, the depth of a unit of n
+// segments is n / kFinGroup^2 batches instead of n / kFinGroup, and the order of every sum is fixed.
+// A record is used only if it carries this launch's epoch and its numbers fit the workspace, so an
+// aborted sweep cannot make this kernel touch memory outside it.
+constexpr int kFinThreads = kHeadDim;   // thread d owns channel d of all G heads
+constexpr int kFinGroup   = 8;
+
+// Merge `count` states at slots slot0, slot0 + step, ...: running (acc, M, z) per head for channel d.
 template <int G>
-__global__ void __launch_bounds__(kConsumerThreads)
-finish_kernel(const int4 *__restrict__ piece_info, const unsigned long long *__restrict__ header,
-              const float *__restrict__ seg, int seg_stride, int seg_slots, float *__restrict__ o_part,
-              float *__restrict__ m_part, float *__restrict__ lse_part, int n_units, int Hkv, int Hq)
+__device__ __forceinline__ void finish_merge_range(const float *__restrict__ seg, int seg_stride, int slot0, int step,
+                                                   int count, float (*s_mz)[2 * G], float *acc, float *M, float *z, int d)
 {
+    constexpr int kB = (G == 8) ? 4 : 8;   // states whose loads are in flight together
+#pragma unroll
+    for (int o = 0; o < G; ++o) { acc[o] = 0.f; M[o] = neg_inf(); z[o] = 0.f; }
+    for (int base = 0; base < count; base += kB) {
+        float av[G][kB];
+#pragma unroll
+        for (int u = 0; u < kB; ++u) {
+            const bool on = base + u < count;
+            const float *sl = seg + (size_t)(slot0 + (on ? base + u : 0) * step) * seg_stride;
+#pragma unroll
+            for (int o = 0; o < G; ++o) av[o][u] = on ? ld_sync_f32(sl + o * kHeadDim + d) : 0.f;
+        }
+        float mz = 0.f;
+        const int u_mine = d / (2 * G), r_mine = d % (2 * G);   // (M, z) pairs of the batch: one word per thread
+        const bool mz_on = u_mine < kB && base + u_mine < count;
+        if (mz_on) mz = ld_sync_f32(seg + (size_t)(slot0 + (base + u_mine) * step) * seg_stride + G * kHeadDim + r_mine);
+        __syncthreads();                       // the previous batch's readers are done with s_mz
+        if (u_mine < kB) s_mz[u_mine][r_mine] = mz_on ? mz : (r_mine & 1 ? 0.f : neg_inf());
+        __syncthreads();
+#pragma unroll
+        for (int o = 0; o < G; ++o) {
+            float Mn = M[o];
+#pragma unroll
+            for (int u = 0; u < kB; ++u) Mn = fmaxf(Mn, s_mz[u][2 * o]);
+            const float Ms = (Mn == neg_inf()) ? 0.f : Mn;
+            const float keep = fast_exp2(M[o] - Ms);   // 0 while nothing has been merged yet
+            z[o] *= keep;
+            acc[o] *= keep;
+#pragma unroll
+            for (int u = 0; u < kB; ++u) {   // fixed order: deterministic
+                const float ew = fast_exp2(s_mz[u][2 * o] - Ms);
+                z[o] = fmaf(s_mz[u][2 * o + 1], ew, z[o]);
+                acc[o] = fmaf(av[o][u], ew, acc[o]);
+            }
+            M[o] = Mn;
+        }
+    }
+}
+
+template <int G>
+__global__ void __launch_bounds__(kFinThreads)
+finish_kernel(const int4 *__restrict__ piece_info, const unsigned long long *__restrict__ header,
+              unsigned long long *__restrict__ counters, float *__restrict__ seg, int seg_stride, int seg_slots,
+              float *__restrict__ o_part, float *__restrict__ m_part, float *__restrict__ lse_part, int n_units,
+              int Hkv, int Hq)
+{
+    static_assert(kFinThreads >= 8 * 2 * G, "one (M, z) word per thread and batch");
+    __shared__ float s_mz[8][2 * G];
+    __shared__ int s_last;
     grid_dependency_wait();
     grid_launch_dependents();
-    const int p = (int)blockIdx.x + 1;      // piece 0 is never a second piece
+    const int d = (int)threadIdx.x;
+    const int p = (int)blockIdx.x + 1;      // piece 0 cannot start inside a unit
     const int n_pieces = (int)(ld_sync_u64(header + kHdrTotals) >> 32);
-    if (p >= n_pieces) return;
-    const int4 rec = ld_sync_int4(piece_info + p);
+    const int4 rec = ld_sync_int4(piece_info + min(p, kMaxSweepCtas + kMaxDynChunks - 1));
     const unsigned long long epoch = ld_sync_u64(header + kHdrLastEpoch);
-    if (rec.x < 0 || rec.w != (int)(unsigned)epoch) return;
+    if (p >= n_pieces || rec.x < 0 || rec.w != (int)(unsigned)epoch) return;
     const int unit = rec.x, first_slot = rec.y, nseg = rec.z;
     if (unit >= n_units || nseg < 2 || first_slot < 0 || (long long)first_slot + nseg > (long long)seg_slots) return;
+    const int k = unit + p - first_slot;    // this piece's segment is the k-th of the unit
+    if (k < 1 || k >= nseg) return;
+    if (k != 1 && (k % kFinGroup) != 0) return;
+    const int group = k / kFinGroup, n_groups = (nseg + kFinGroup - 1) / kFinGroup;
+    const int seg0 = group * kFinGroup;
     const size_t out_row = (size_t)(unit / Hkv) * Hq + (size_t)(unit % Hkv) * G;
-    merge_segments<G, kConsumerThreads>(seg, seg_stride, first_slot, 1, nseg, out_row, o_part, m_part, lse_part,
-                                        (int)threadIdx.x);
+    const float kLn2 = 0.6931471805599453f;
+
+    float acc[G], M[G], z[G];
+    auto write_final = [&]() {
+#pragma unroll
+        for (int o = 0; o < G; ++o) {
+            const bool empty = (M[o] == neg_inf());
+            o_part[(out_row + o) * kHeadDim + d] = empty ? 0.f : acc[o] / z[o];
+            if (d == 0) {
+                m_part[out_row + o] = empty ? neg_inf() : M[o] * kLn2;
+                lse_part[out_row + o] = empty ? neg_inf() : (M[o] + log2f(z[o])) * kLn2;
+            }
+        }
+    };
+    finish_merge_range<G>(seg, seg_stride, first_slot + seg0, 1, min(kFinGroup, nseg - seg0), s_mz, acc, M, z, d);
+    if (n_groups == 1) { write_final(); return; }
+
+    // the group's partial state replaces the group's first segment (which only this CTA reads)
+    float *slot = seg + (size_t)(first_slot + seg0) * seg_stride;
+#pragma unroll
+    for (int o = 0; o < G; ++o) {
+        __stcg(slot + o * kHeadDim + d, acc[o]);
+        if (d == 0) { __stcg(slot + G * kHeadDim + 2 * o, M[o]); __stcg(slot + G * kHeadDim + 2 * o + 1, z[o]); }
+    }
+    __syncthreads();
+    if (d == 0) {
+        __threadfence();
+        s_last = (epoch_arrive(counters + unit, epoch) == (unsigned)n_groups) ? 1 : 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    finish_merge_range<G>(seg, seg_stride, first_slot, kFinGroup, n_groups, s_mz, acc, M, z, d);
+    write_final();
 }
 
 // ------------------------------------------------------------------ bounded-wait self-test
@@ -785,6 +911,7 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
     unsigned long long *header = reinterpret_cast<unsigned long long *>(ws + wsl.header_off);
     int *prefix = reinterpret_cast<int *>(ws + wsl.prefix_off);
     int4 *piece_info = reinterpret_cast<int4 *>(ws + wsl.piece_off);
+    unsigned long long *counters = reinterpret_cast<unsigned long long *>(ws + wsl.counter_off);
     float *seg = reinterpret_cast<float *>(ws + wsl.seg_off);
     const int n_entries = P.batch * P.max_shards;
     const size_t smem = sizeof(SweepSmem<G>) + 1024;
@@ -812,9 +939,9 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
     if (ev1) cudaEventRecord(ev1, st);
     if (e != cudaSuccess) { snprintf(msg, msg_len, "sweep_kernel launch: %s", cudaGetErrorString(e)); return -5; }
     *launches += 1;
-    // one CTA per piece that can be a unit's second piece
-    e = launch_pdl(finish_kernel<G>, dim3(n_ctas + kMaxDynChunks - 1), dim3(kConsumerThreads), 0, st,
-                   (const int4 *)piece_info, (const unsigned long long *)header, (const float *)seg, wsl.seg_stride,
+    // one CTA per piece that can start inside a unit
+    e = launch_pdl(finish_kernel<G>, dim3(n_ctas + kMaxDynChunks - 1), dim3(kFinThreads), 0, st,
+                   (const int4 *)piece_info, (const unsigned long long *)header, counters, seg, wsl.seg_stride,
                    (int)wsl.seg_slots, o, m, l, n_entries * P.num_kv_heads, P.num_kv_heads, P.num_q_heads);
     if (e != cudaSuccess) { snprintf(msg, msg_len, "finish_kernel launch: %s", cudaGetErrorString(e)); return -5; }
     *launches += 1;

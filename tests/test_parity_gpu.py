@@ -31,8 +31,10 @@ def run(w, flags=0, null_table=False):
 
 # (flags, number of KV heads): the unit kernel is the default; the head-parallel kernel is opt-in and needs
 # KV heads in groups of eight; the plain-load kernel is the validation aid
+# "draw": the unit kernel with its drawn-chunk tail forced on (by default only long sweeps use it)
 KERNELS = [pytest.param((qf.QF_FLAG_HEAD_PARALLEL, 8), id="headpar"), pytest.param((0, 8), id="unit8"),
-           pytest.param((0, 2), id="unit2"), pytest.param((qf.QF_FLAG_SIMPLE_KERNEL, 2), id="simple")]
+           pytest.param((0, 2), id="unit2"), pytest.param((qf.QF_FLAG_SIMPLE_KERNEL, 2), id="simple"),
+           pytest.param((qf.QF_FLAG_DRAW_ALWAYS, 8), id="draw8"), pytest.param((qf.QF_FLAG_DRAW_ALWAYS, 2), id="draw2")]
 
 
 # T1: every short length, both group sizes, shuffled table: tail-page masking, first-tile guard
@@ -232,7 +234,8 @@ def test_medium_ragged_batch(G, seed, flags):
     assert dw.status() == 0
 
 
-@pytest.mark.parametrize("Hkv,flags", [(2, 0), (8, 0), (8, qf.QF_FLAG_HEAD_PARALLEL), (16, qf.QF_FLAG_HEAD_PARALLEL)])
+@pytest.mark.parametrize("Hkv,flags", [(2, 0), (8, 0), (8, qf.QF_FLAG_HEAD_PARALLEL), (16, qf.QF_FLAG_HEAD_PARALLEL),
+                                       (2, qf.QF_FLAG_DRAW_ALWAYS), (8, qf.QF_FLAG_DRAW_ALWAYS)])
 def test_long_single_request_many_segments(Hkv, flags):
     # one request whose single shard is split over every SM by the balanced schedule
     L = 150_001 if Hkv <= 8 else 40_001
@@ -251,6 +254,40 @@ def test_small_configs_elementwise():
         T.compare_all(dws, w, tag=w.name + "/simple")
         dwh = run(w, qf.QF_FLAG_HEAD_PARALLEL)
         T.compare_all(dwh, w, tag=w.name + "/headpar")
+
+
+# The schedule of the unit kernel: equal static slices, then chunks of halving size drawn from a counter;
+# units cut by piece boundaries are merged by the finish kernel.  Totals from just above the smallest
+# sweep that draws (two stage units per SM) up to the size at which drawing is on by default, with units
+# much shorter than a chunk, about a chunk, and much longer; the result must not depend on the flag
+# beyond fp32 summation order, and both must match the oracle element by element.
+@pytest.mark.parametrize("B,L,shard,Hkv,G", [
+    (3, 2100, 2100, 8, 4),        # ~400 stage units: a few per SM
+    (40, 700, 130, 8, 2),         # units of one or two stages: most chunks hold several whole units
+    (6, 9000, 1024, 8, 4),        # units of 8 stages
+    (2, 60_000, 60_000, 8, 2),    # two very long units per KV head: every unit cut many times
+    (10, 20_000, 4096, 8, 4),     # ~12,600 stage units: drawing is on by default
+    (5, 33_000, 7000, 2, 8),      # G = 8 (two epilogue rounds), few KV heads
+])
+def test_drawn_chunk_schedule(B, L, shard, Hkv, G):
+    rng = np.random.default_rng(B * 1000 + L)
+    lens = [int(x) for x in rng.integers(L // 2, L + 1, size=B)]
+    w = wl.make_workload("draw", lens, [wl.fixed_shards(x, shard) for x in lens], Hkv * G, Hkv, seed=L + G,
+                         pool_factor=1.3, poison_unused=True, poison_tails=True)
+    res = {}
+    for flags in (0, qf.QF_FLAG_DRAW_ALWAYS):
+        dw = run(w, flags)
+        T.compare_all(dw, w, tag=f"flags={flags}")
+        assert dw.status() == 0
+        res[flags] = [r.copy() for r in dw.results()]
+        # replays of the same launch give the same bits (who draws which chunk varies, the result must not)
+        for _ in range(3):
+            dw.poison_outputs()
+            dw.step()
+            for x, y in zip(res[flags], dw.results()):
+                assert np.array_equal(x, y)
+    for x, y in zip(res[0], res[qf.QF_FLAG_DRAW_ALWAYS]):
+        assert np.allclose(x, y, rtol=0, atol=T.ENG_OUT, equal_nan=True)
 
 
 # T9: run-to-run determinism and canaries around the outputs
@@ -343,7 +380,7 @@ def test_a_wait_that_cannot_be_satisfied_times_out_and_leaves_the_context_usable
     T.compare_all(dw, w)
 
 
-@pytest.mark.parametrize("flags", [0, qf.QF_FLAG_HEAD_PARALLEL])
+@pytest.mark.parametrize("flags", [0, qf.QF_FLAG_HEAD_PARALLEL, qf.QF_FLAG_DRAW_ALWAYS])
 def test_cuda_graph_replay_with_new_queries(flags):
     # a captured decode step replayed with fresh queries: every replay must behave like a fresh launch
     # (the scratch words that must "start at zero" are tagged per launch, also under replay)
@@ -369,7 +406,7 @@ def test_cuda_graph_replay_with_new_queries(flags):
         assert dw.status() == 0
 
 
-@pytest.mark.parametrize("seed", list(range(24)))
+@pytest.mark.parametrize("seed", list(range(32)))
 def test_randomized_shapes_and_ranges(seed):
     # random batch, head counts, group size, lengths, unaligned / overlapping / empty shard ranges, pool slack
     rng = np.random.default_rng(1000 + seed)
@@ -391,7 +428,8 @@ def test_randomized_shapes_and_ranges(seed):
                 a, b = sorted(int(x) for x in rng.integers(-3, L + 5, size=2))
                 rr.append((a, b))
         ranges.append(rr)
-    flags = int(rng.choice([0, 0, qf.QF_FLAG_HEAD_PARALLEL, qf.QF_FLAG_CHECK_BOUNDS]))
+    flags = int(rng.choice([0, qf.QF_FLAG_DRAW_ALWAYS, qf.QF_FLAG_HEAD_PARALLEL, qf.QF_FLAG_CHECK_BOUNDS,
+                            qf.QF_FLAG_DRAW_ALWAYS | qf.QF_FLAG_CHECK_BOUNDS]))
     w = wl.make_workload("fuzz", lens, ranges, Hkv * G, Hkv, seed=seed, pool_factor=float(rng.choice([1.0, 1.5])),
                          poison_unused=True, poison_tails=True, max_pages_per_req=max(1, (max(lens) + 15) // 16 + 2))
     dw = run(w, flags)
