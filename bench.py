@@ -2,7 +2,8 @@
 """Benchmark of the Q-First cache-side decode path on B200.
 
 A step is one pass of the whole hot path over one batch of synthetic input:
-the sweep kernel (plan, stream, segment merge: shard states) and the combine kernel.  The default
+the sweep kernel (plan, stream, warp merge: shard states or segments of them), the finish kernel
+(merges the shards that the schedule cut into segments) and the combine kernel.  The default
 workload is the Qwen3-4B-shaped batched decode (32 requests, 32 q / 8 kv heads,
 ragged contexts in [1,024, 36,480], 16-token pages in a shuffled block table,
 4,096-token shards), the configuration the headline metric is quoted on.
@@ -33,7 +34,7 @@ if str(ROOT) not in sys.path:
 METRIC = "decode-attention KV GB/s and % of B200 HBM peak (Qwen3-4B shape, batched)"
 # dram__bytes_read.sum + dram__bytes_write.sum of one sweep-kernel launch, from the committed ncu summaries of
 # the Qwen3-4B-shaped and one-million-token workloads (seed 0)
-NCU_TRAFFIC_BYTES = {3: 2013172000 + 5599744, 4: 4295371264 + 233728}
+NCU_TRAFFIC_BYTES = {3: 2013151000 + 5875456, 4: 4295394816 + 605952}
 FALLBACK_HBM_GBS = 6650.0
 DATASHEET_HBM_GBS = 8000.0
 

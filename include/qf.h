@@ -97,10 +97,6 @@ enum {
 enum {
     QF_FLAG_CHECK_BOUNDS  = 1, /* range-check page indices on the device           */
     QF_FLAG_SIMPLE_KERNEL = 2, /* use the plain-load sweep kernel (validation aid) */
-    QF_FLAG_HEAD_PARALLEL = 4, /* use the head-parallel sweep kernel (needs Hkv a multiple
-                                  of 8 and G <= 4, else ignored): one page of eight KV
-                                  heads per ring stage, no cross-warp merges; faster when
-                                  shards are short (a few hundred tokens to ~2,000)      */
     QF_FLAG_DRAW_ALWAYS   = 8  /* default sweep kernel only: hand out the tail of the work
                                   as drawn chunks however short the sweep is (by default
                                   only sweeps long enough to gain from it do).  Same
@@ -138,8 +134,9 @@ const char *qf_strerror(int status);
 /*
  * Bytes of device scratch qf_decode_partial needs for these parameters
  * (0 if the parameters are invalid).  The scratch holds the sweep plan
- * (prefix sums over shards), per-CTA segment states that are merged into the
- * per-shard states, and a status word.  Contents need not be initialised.
+ * (prefix sums over shards), one record per piece of the schedule, segment
+ * states that are merged into the per-shard states, and a status word.
+ * Contents need not be initialised.
  * The pointer passed later must be 256-byte aligned.
  */
 size_t qf_workspace_bytes(const qf_params *p);
@@ -153,7 +150,11 @@ size_t qf_workspace_bytes(const qf_params *p);
  *     lse_part[b,s,h] = log Z(S).
  * Every one of the B*S slots is written (empty: 0, -inf, -inf).
  * All pointers are device pointers; block_table may be NULL (identity).
- * K/V pool pointers must be 128-byte aligned.  Enqueues on cuda_stream.
+ * K/V pool pointers must be 128-byte aligned.  Enqueues on cuda_stream: the
+ * sweep kernel, then a small finish kernel that merges the (shard, KV head)
+ * units the schedule cut into segments; a one-CTA plan kernel goes first when
+ * batch * max_shards > 2,048.  The outputs are complete when the last of them
+ * has run.
  */
 int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache,
                       const int32_t *block_table, const int32_t *seq_lens,

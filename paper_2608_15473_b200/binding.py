@@ -28,7 +28,6 @@ QF_STATIC_SCRATCH_BYTES = 8 << 20
 
 QF_FLAG_CHECK_BOUNDS = 1
 QF_FLAG_SIMPLE_KERNEL = 2
-QF_FLAG_HEAD_PARALLEL = 4
 QF_FLAG_DRAW_ALWAYS = 8
 
 QF_STATUS_BAD_PAGE = 1

@@ -11,7 +11,6 @@
 #include "qf_common.cuh"
 #include "qf_simple.cuh"
 #include "qf_sweep.cuh"
-#include "qf_sweep_hp.cuh"
 
 namespace {
 
@@ -168,9 +167,9 @@ int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache, c
     }
 
     int launches = 0;
-    rc = qf::launch_sweep_any(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P,
-                              (char *)workspace, wsl, sms, epoch, (p->flags & QF_FLAG_HEAD_PARALLEL) != 0, st,
-                              g_prof_start, g_prof_stop, g_cuda_msg, sizeof g_cuda_msg, &launches);
+    rc = qf::launch_sweep(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P,
+                          (char *)workspace, wsl, sms, epoch, st, g_prof_start, g_prof_stop, g_cuda_msg,
+                          sizeof g_cuda_msg, &launches);
     g_last_launches = launches;
     return rc;
 }

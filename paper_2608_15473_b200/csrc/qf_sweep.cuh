@@ -83,26 +83,22 @@ inline WorkspaceLayout workspace_layout(int batch, int max_shards, int num_kv_he
     L.piece_off = up(L.counter_off + entries * num_kv_heads * sizeof(unsigned long long));
     L.seg_off = up(L.piece_off + (size_t)(kMaxSweepCtas + kMaxDynChunks) * sizeof(int4));
     L.seg_stride = seg_stride_floats(G);
-    // unit kernel: slot = unit + piece; head-parallel kernel: two slot groups of eight heads per CTA
-    const size_t unit_slots = entries * num_kv_heads + (size_t)kMaxSweepCtas + (size_t)kMaxDynChunks;
-    const size_t hp_slots = (num_kv_heads % 8 == 0 && G <= 4) ? (size_t)kMaxSweepCtas * 2 * 8 : 0;
-    const size_t slots = unit_slots > hp_slots ? unit_slots : hp_slots;
+    // a cut unit's segment lives in slot (unit + piece): both grow along the unit space, so slots are unique
+    const size_t slots = entries * num_kv_heads + (size_t)kMaxSweepCtas + (size_t)kMaxDynChunks;
     L.seg_slots = slots;
     L.total = up(L.seg_off + slots * L.seg_stride * sizeof(float));
     return L;
 }
 
-// Work units of entry e = (request, shard), all KV heads together.  hp_groups == 0: stage units of
-// kPagesPerStage pages per KV head (unit kernel); hp_groups > 0: pages per group of eight KV heads
-// (head-parallel kernel).
+// Work units of entry e = (request, shard), all KV heads together: stage units of kPagesPerStage pages
+// per KV head.
 __device__ __forceinline__ int entry_units(const int *__restrict__ seq_lens, const int *__restrict__ shard_ranges,
-                                           int e, int max_shards, int num_kv_heads, int hp_groups)
+                                           int e, int max_shards, int num_kv_heads)
 {
     int beg, end;
     clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[e / max_shards], beg, end);
     if (end <= beg) return 0;
     const int npages = ((end - 1) >> 4) - (beg >> 4) + 1;
-    if (hp_groups > 0) return npages * hp_groups;
     return ((npages + kPagesPerStage - 1) / kPagesPerStage) * num_kv_heads;
 }
 
@@ -181,14 +177,14 @@ __device__ __forceinline__ void piece_range(const PieceGrid &g, int n_ctas, int 
 // prefix[e] = number of stage units before entry e = b*S + s, left in scratch.
 __global__ void __launch_bounds__(1024)
 plan_kernel(const int *__restrict__ seq_lens, const int *__restrict__ shard_ranges, int *__restrict__ prefix,
-            int n_entries, int max_shards, int num_kv_heads, int hp_groups)
+            int n_entries, int max_shards, int num_kv_heads)
 {
     __shared__ int warp_sums[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int carry = 0;
     for (int base = 0; base < n_entries; base += 1024) {
         const int e = base + tid;
-        const int cnt = (e < n_entries) ? entry_units(seq_lens, shard_ranges, e, max_shards, num_kv_heads, hp_groups) : 0;
+        const int cnt = (e < n_entries) ? entry_units(seq_lens, shard_ranges, e, max_shards, num_kv_heads) : 0;
         int x = cnt;  // inclusive scan within the warp
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -243,75 +239,6 @@ struct SweepSmem {
     int prefix[kMaxSmemEntries + 1];
 };
 
-// Merge segments [first, first+nseg) of one (shard, KV head) unit into its final state.
-// Called by the NT threads (a warp or all consumer warps) that arrived last; fixed order, so deterministic.
-// A thread owns outputs idx = tid + k*NT and handles two of them at a time; per pair it walks the segments
-// in batches of eight with all of a batch's loads in flight together (one L2 round trip per batch) and a
-// running maximum, so a unit cut into up to eight segments costs one round trip per output pair.
-template <int G, int NT>
-__device__ __forceinline__ void merge_segments(const float *__restrict__ seg, int seg_stride, int first_slot,
-                                               int slot_step, int nseg, size_t out_row, float *__restrict__ o_part,
-                                               float *__restrict__ m_part, float *__restrict__ lse_part, int tid)
-{
-    const float kLn2 = 0.6931471805599453f;
-    constexpr int kBatch = 8;   // segments whose loads are in flight together
-    constexpr int kPair = 2;    // outputs a thread merges together
-    for (int idx0 = tid; idx0 < G * kHeadDim; idx0 += kPair * NT) {
-        float M[kPair], z[kPair], acc[kPair];
-        int head[kPair], d[kPair];
-        bool on_o[kPair];
-#pragma unroll
-        for (int o = 0; o < kPair; ++o) {
-            const int idx = idx0 + o * NT;
-            on_o[o] = idx < G * kHeadDim;
-            head[o] = on_o[o] ? idx >> 7 : 0;
-            d[o] = idx & 127;
-            M[o] = neg_inf(); z[o] = 0.f; acc[o] = 0.f;
-        }
-        for (int base = 0; base < nseg; base += kBatch) {
-            float mv[kPair][kBatch], zv[kPair][kBatch], av[kPair][kBatch];
-#pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                const bool on = base + u < nseg;
-                const float *sl = seg + (size_t)(first_slot + (on ? base + u : 0) * slot_step) * seg_stride;
-#pragma unroll
-                for (int o = 0; o < kPair; ++o) {
-                    mv[o][u] = on ? ld_sync_f32(sl + G * kHeadDim + 2 * head[o]) : neg_inf();
-                    zv[o][u] = on ? ld_sync_f32(sl + G * kHeadDim + 2 * head[o] + 1) : 0.f;
-                    av[o][u] = on ? ld_sync_f32(sl + head[o] * kHeadDim + d[o]) : 0.f;
-                }
-            }
-#pragma unroll
-            for (int o = 0; o < kPair; ++o) {
-                float Mn = M[o];
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u) Mn = fmaxf(Mn, mv[o][u]);
-                const float Ms = (Mn == neg_inf()) ? 0.f : Mn;
-                const float keep = fast_exp2(M[o] - Ms);   // 0 while nothing has been merged yet
-                z[o] *= keep;
-                acc[o] *= keep;
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u) {   // fixed order: deterministic
-                    const float ew = fast_exp2(mv[o][u] - Ms);
-                    z[o] = fmaf(zv[o][u], ew, z[o]);
-                    acc[o] = fmaf(av[o][u], ew, acc[o]);
-                }
-                M[o] = Mn;
-            }
-        }
-#pragma unroll
-        for (int o = 0; o < kPair; ++o) {
-            if (!on_o[o]) continue;
-            const bool empty = (M[o] == neg_inf());
-            o_part[(out_row + head[o]) * kHeadDim + d[o]] = empty ? 0.f : acc[o] / z[o];
-            if (d[o] == 0) {
-                m_part[out_row + head[o]] = empty ? neg_inf() : M[o] * kLn2;
-                lse_part[out_row + head[o]] = empty ? neg_inf() : (M[o] + log2f(z[o])) * kLn2;
-            }
-        }
-    }
-}
-
 template <int G>
 __global__ void __launch_bounds__(kSweepThreads, 1)
 sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
@@ -362,7 +289,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
         for (int base = 0; base < n_entries; base += kConsumerThreads) {
             const int e = base + tid;
             const int cnt = (tid < kConsumerThreads && e < n_entries)
-                                ? entry_units(seq_lens, shard_ranges, e, S, Hkv, 0) : 0;
+                                ? entry_units(seq_lens, shard_ranges, e, S, Hkv) : 0;
             int x = cnt;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
@@ -926,7 +853,7 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
     *launches = 0;
     const int *global_prefix = nullptr;
     if (n_entries > kMaxSmemEntries) {
-        plan_kernel<<<1, 1024, 0, st>>>(sl, sr, prefix, n_entries, P.max_shards, P.num_kv_heads, 0);
+        plan_kernel<<<1, 1024, 0, st>>>(sl, sr, prefix, n_entries, P.max_shards, P.num_kv_heads);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) { snprintf(msg, msg_len, "plan_kernel launch: %s", cudaGetErrorString(e)); return -5; }
         global_prefix = prefix;

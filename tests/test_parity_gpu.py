@@ -29,10 +29,9 @@ def run(w, flags=0, null_table=False):
     return dw
 
 
-# (flags, number of KV heads): the unit kernel is the default; the head-parallel kernel is opt-in and needs
-# KV heads in groups of eight; the plain-load kernel is the validation aid
+# (flags, number of KV heads): the default kernel with 8 and 2 KV heads; the plain-load kernel is the validation aid
 # "draw": the unit kernel with its drawn-chunk tail forced on (by default only long sweeps use it)
-KERNELS = [pytest.param((qf.QF_FLAG_HEAD_PARALLEL, 8), id="headpar"), pytest.param((0, 8), id="unit8"),
+KERNELS = [pytest.param((0, 16), id="unit16"), pytest.param((0, 8), id="unit8"),
            pytest.param((0, 2), id="unit2"), pytest.param((qf.QF_FLAG_SIMPLE_KERNEL, 2), id="simple"),
            pytest.param((qf.QF_FLAG_DRAW_ALWAYS, 8), id="draw8"), pytest.param((qf.QF_FLAG_DRAW_ALWAYS, 2), id="draw2")]
 
@@ -234,8 +233,7 @@ def test_medium_ragged_batch(G, seed, flags):
     assert dw.status() == 0
 
 
-@pytest.mark.parametrize("Hkv,flags", [(2, 0), (8, 0), (8, qf.QF_FLAG_HEAD_PARALLEL), (16, qf.QF_FLAG_HEAD_PARALLEL),
-                                       (2, qf.QF_FLAG_DRAW_ALWAYS), (8, qf.QF_FLAG_DRAW_ALWAYS)])
+@pytest.mark.parametrize("Hkv,flags", [(2, 0), (8, 0), (16, 0), (2, qf.QF_FLAG_DRAW_ALWAYS), (8, qf.QF_FLAG_DRAW_ALWAYS)])
 def test_long_single_request_many_segments(Hkv, flags):
     # one request whose single shard is split over every SM by the balanced schedule
     L = 150_001 if Hkv <= 8 else 40_001
@@ -252,8 +250,8 @@ def test_small_configs_elementwise():
         T.compare_all(dw, w, tag=w.name)
         dws = run(w, qf.QF_FLAG_SIMPLE_KERNEL)
         T.compare_all(dws, w, tag=w.name + "/simple")
-        dwh = run(w, qf.QF_FLAG_HEAD_PARALLEL)
-        T.compare_all(dwh, w, tag=w.name + "/headpar")
+        dwd = run(w, qf.QF_FLAG_DRAW_ALWAYS)
+        T.compare_all(dwd, w, tag=w.name + "/draw")
 
 
 # The schedule of the unit kernel: equal static slices, then chunks of halving size drawn from a counter;
@@ -354,7 +352,7 @@ def test_full_size_configs_sampled(cfg, seed):
     assert dw.status() == 0
 
 
-@pytest.mark.parametrize("Hkv,flags", [(2, 0), (8, 0), (8, qf.QF_FLAG_HEAD_PARALLEL)])
+@pytest.mark.parametrize("Hkv,flags", [(2, 0), (8, 0), (8, qf.QF_FLAG_DRAW_ALWAYS)])
 def test_many_entries_plan_in_scratch(Hkv, flags):
     # more (request, shard) pairs than the in-kernel plan holds: the separate plan kernel path
     rng = np.random.default_rng(41)
@@ -380,7 +378,7 @@ def test_a_wait_that_cannot_be_satisfied_times_out_and_leaves_the_context_usable
     T.compare_all(dw, w)
 
 
-@pytest.mark.parametrize("flags", [0, qf.QF_FLAG_HEAD_PARALLEL, qf.QF_FLAG_DRAW_ALWAYS])
+@pytest.mark.parametrize("flags", [0, qf.QF_FLAG_DRAW_ALWAYS])
 def test_cuda_graph_replay_with_new_queries(flags):
     # a captured decode step replayed with fresh queries: every replay must behave like a fresh launch
     # (the scratch words that must "start at zero" are tagged per launch, also under replay)
@@ -428,7 +426,7 @@ def test_randomized_shapes_and_ranges(seed):
                 a, b = sorted(int(x) for x in rng.integers(-3, L + 5, size=2))
                 rr.append((a, b))
         ranges.append(rr)
-    flags = int(rng.choice([0, qf.QF_FLAG_DRAW_ALWAYS, qf.QF_FLAG_HEAD_PARALLEL, qf.QF_FLAG_CHECK_BOUNDS,
+    flags = int(rng.choice([0, qf.QF_FLAG_DRAW_ALWAYS, qf.QF_FLAG_CHECK_BOUNDS,
                             qf.QF_FLAG_DRAW_ALWAYS | qf.QF_FLAG_CHECK_BOUNDS]))
     w = wl.make_workload("fuzz", lens, ranges, Hkv * G, Hkv, seed=seed, pool_factor=float(rng.choice([1.0, 1.5])),
                          poison_unused=True, poison_tails=True, max_pages_per_req=max(1, (max(lens) + 15) // 16 + 2))
