@@ -188,7 +188,9 @@ int launch_combine(const float *o_part, const float *lse_part, const int32_t *sh
     const qf::DevParams P = dev_params(p);
     const long long bh = (long long)p->batch * p->num_q_heads;
     const unsigned blocks = (unsigned)((bh + qf::kCombineWarps - 1) / qf::kCombineWarps);
-    cudaError_t e = qf::launch_pdl(qf::combine_kernel, dim3(blocks), dim3(qf::kCombineWarps * 32), 0,
+    auto kernel = p->max_shards <= 4 ? qf::combine_kernel<4> : p->max_shards <= 8 ? qf::combine_kernel<8>
+                                                                                  : qf::combine_kernel<16>;
+    cudaError_t e = qf::launch_pdl(kernel, dim3(blocks), dim3(qf::kCombineWarps * 32), 0,
                                    (cudaStream_t)cuda_stream, o_part, lse_part, shard_counts, (const uint16_t *)q,
                                    (const uint16_t *)k_new, (const uint16_t *)v_new, out, lse, p->batch,
                                    p->num_q_heads, p->num_kv_heads, p->max_shards, P.sm_scale);

@@ -16,6 +16,9 @@ namespace qf {
 constexpr int kCombineWarps = 4;
 
 // q, k_new, v_new: nullptr = no current token.  k_new, v_new: bf16 [B, Hkv, D].
+// kCombineBatch: shard vectors in flight per lane (the host picks the smallest that covers max_shards,
+// up to 16: fewer registers, more resident warps when shards are few).
+template <int kCombineBatch>
 __global__ void __launch_bounds__(kCombineWarps * 32)
 combine_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_part,
                const int *__restrict__ shard_counts, const uint16_t *__restrict__ q,
@@ -29,9 +32,6 @@ combine_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_p
     const long long bh = (long long)blockIdx.x * kCombineWarps + (threadIdx.x >> 5);
     if (bh >= (long long)batch * num_q_heads) return;
     const int b = (int)(bh / num_q_heads), h = (int)(bh % num_q_heads);
-    int ns = shard_counts ? shard_counts[b] : max_shards;
-    ns = min(max(ns, 0), max_shards);
-
     // the current token, if any: its score against this head's query and its value row
     float s_self = neg_inf();
     float4 v_self = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -51,42 +51,57 @@ combine_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_p
         v_self = make_float4(bf16lo_to_f32(vw.x), bf16hi_to_f32(vw.x), bf16lo_to_f32(vw.y), bf16hi_to_f32(vw.y));
     }
 
+    // Everything the merge reads is requested before anything is waited for: the shard count, the first 32
+    // log Z values (lane s holds shard s) and the first kCombineBatch shard vectors go out together, one
+    // round trip to L2 for the usual shard counts.  Slots at or beyond the shard count exist (the arrays
+    // have max_shards slots per request) but may hold anything: they are masked below, never multiplied.
     const float *lrow = lse_part + ((size_t)b * max_shards) * num_q_heads + h;
+    const float *obase = o_part + (((size_t)b * max_shards) * num_q_heads + h) * kHeadDim + lane * 4;
+    const size_t ostride = (size_t)num_q_heads * kHeadDim;
+    const float ls_first = (lane < max_shards) ? lrow[(size_t)lane * num_q_heads] : neg_inf();
+    float4 o[kCombineBatch];
+#pragma unroll
+    for (int u = 0; u < kCombineBatch; ++u)
+        o[u] = (u < max_shards) ? *reinterpret_cast<const float4 *>(obase + (size_t)u * ostride)
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+    bool loaded = true;   // o[] holds shards 0 .. kCombineBatch-1
+    int ns = shard_counts ? shard_counts[b] : max_shards;
+    ns = min(max(ns, 0), max_shards);
+
     // M = max over operands of log Z; lanes stride over shards
     float M = s_self;
-    for (int s = lane; s < ns; s += 32) M = fmaxf(M, lrow[(size_t)s * num_q_heads]);
+    if (lane < ns) M = fmaxf(M, ls_first);
+    for (int s = lane + 32; s < ns; s += 32) M = fmaxf(M, lrow[(size_t)s * num_q_heads]);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
 
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float wsum = 0.f;
     if (M != neg_inf()) {
-        const float *obase = o_part + (((size_t)b * max_shards) * num_q_heads + h) * kHeadDim + lane * 4;
-        const size_t ostride = (size_t)num_q_heads * kHeadDim;
         for (int base = 0; base < ns; base += 32) {
             // lane s holds shard (base+s)'s weight e^{lse_s - M}: in (0, 1], cannot overflow; 0 for empty shards
             const int sl = base + lane;
-            const float ls = (sl < ns) ? lrow[(size_t)sl * num_q_heads] : neg_inf();
+            float ls = neg_inf();
+            if (sl < ns) ls = (base == 0) ? ls_first : lrow[(size_t)sl * num_q_heads];
             const float w = (ls == neg_inf()) ? 0.f : expf(ls - M);
             wsum += w;
             const int cnt = min(32, ns - base);
-            for (int j = 0; j < cnt; j += 4) {
-                float wj[4];
-                float4 o[4];
+            for (int j = 0; j < cnt; j += kCombineBatch) {
+                if (!loaded) {
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {   // four independent 512-byte reads in flight
-                    wj[u] = __shfl_sync(0xffffffffu, w, (j + u) & 31);
-                    if (j + u >= cnt) wj[u] = 0.f;
-                    o[u] = (j + u < cnt) ? *reinterpret_cast<const float4 *>(obase + (size_t)(base + j + u) * ostride)
-                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int u = 0; u < kCombineBatch; ++u)   // independent 512-byte reads in flight together
+                        o[u] = (j + u < cnt) ? *reinterpret_cast<const float4 *>(obase + (size_t)(base + j + u) * ostride)
+                                             : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
+                loaded = false;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (wj[u] != 0.f) {         // an empty shard's vector is loaded but never used
-                        acc.x = fmaf(wj[u], o[u].x, acc.x);
-                        acc.y = fmaf(wj[u], o[u].y, acc.y);
-                        acc.z = fmaf(wj[u], o[u].z, acc.z);
-                        acc.w = fmaf(wj[u], o[u].w, acc.w);
+                for (int u = 0; u < kCombineBatch; ++u) {
+                    const float wu = __shfl_sync(0xffffffffu, w, (j + u) & 31);
+                    if (j + u < cnt && wu != 0.f) {   // an empty shard's vector is loaded but never used
+                        acc.x = fmaf(wu, o[u].x, acc.x);
+                        acc.y = fmaf(wu, o[u].y, acc.y);
+                        acc.z = fmaf(wu, o[u].z, acc.z);
+                        acc.w = fmaf(wu, o[u].w, acc.w);
                     }
                 }
             }
