@@ -7,21 +7,25 @@
 //
 //   plan      every CTA turns (seq_lens, shard_ranges) into a prefix sum over "stage
 //             units" (8 pages = 128 tokens of one KV head of one shard) in shared
-//             memory and takes an equal contiguous slice of the unit space (no atomics,
-//             no work queue).  Batches with more than kMaxSmemEntries (request, shard)
-//             pairs use a separate plan kernel that leaves the prefix in scratch.
-//   stream    a producer warp walks the slice, looks pages up in the block table and
+//             memory.  The unit space is cut into pieces (PieceGrid): one equal static
+//             slice per CTA over the first nine tenths, and chunks of halving size over
+//             the rest, which CTAs draw from a counter as they run out of work.  Batches
+//             with more than kMaxSmemEntries (request, shard) pairs use a separate plan
+//             kernel that leaves the prefix in scratch (and static slices only).
+//   stream    a producer warp walks its pieces, looks pages up in the block table and
 //             issues one 4 KB TMA box per K or V page (128B-swizzled) into a 3-stage shared-memory ring;
 //             8 consumer warps each take one page of a stage: S = K Q^T on tensor cores
 //             (tokens on M, the group's heads on N), fp32 online softmax, P split into
 //             bf16 hi+lo, O^T += V^T P^T.
-//   merge     a slice boundary inside a (shard, KV head) unit leaves segment states in
-//             scratch; the last CTA to finish a segment of that unit (epoch-tagged
-//             arrival counter) merges them in fixed order into o_part/m_part/lse_part.
-//             Empty shards get (0, -inf, -inf) from the consumer warps' prologue.
+//   merge     at a segment end the eight warps' states merge through shared memory into
+//             the shard's state, or, if a piece boundary cut the (shard, KV head) unit,
+//             into a segment slot of the scratch that the finish kernel (qf_finish.cuh)
+//             merges after the sweep.  Empty shards get (0, -inf, -inf) from the consumer
+//             warps' prologue.
 //
 // All waits are bounded: a wait that runs out sets QF_STATUS_TIMEOUT, raises a
-// CTA-wide abort flag and every warp leaves.  No CTA ever waits for another CTA.
+// CTA-wide abort flag and every warp leaves.  No CTA ever waits for another CTA
+// (drawing a chunk is one atomic add; it never blocks on another CTA's progress).
 #pragma once
 
 #include <cuda.h>
@@ -34,6 +38,7 @@
 
 #include "qf_common.cuh"
 #include "qf_page_math.cuh"
+#include "qf_finish.cuh"
 
 namespace qf {
 
@@ -625,128 +630,6 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     }
 }
 
-// ------------------------------------------------------------------ finish kernel
-// Merges the units that piece boundaries cut into segments, after the sweep (not inside it, by whoever
-// arrives last at a counter: a merge is a few round trips to L2, several microseconds each while the
-// memory system is saturated, and it would land on the CTAs that are already late).
-//
-// CTA p looks at the record piece p left.  If the piece starts inside a unit, its segment is the k-th of
-// that unit (k >= 1).  Segments are merged in groups of kFinGroup: the CTAs with k == 1 or k a multiple of
-// kFinGroup lead a group, the others exit.  A unit of one group is finished by its leader.  Otherwise each
-// leader writes its group's partial state over the group's first slot and arrives at the unit's counter;
-// the leader that arrives last merges the partials.  Nobody waits for anybody, the depth of a unit of n
-// segments is n / kFinGroup^2 batches instead of n / kFinGroup, and the order of every sum is fixed.
-// A record is used only if it carries this launch's epoch and its numbers fit the workspace, so an
-// aborted sweep cannot make this kernel touch memory outside it.
-constexpr int kFinThreads = kHeadDim;   // thread d owns channel d of all G heads
-constexpr int kFinGroup   = 8;
-
-// Merge `count` states at slots slot0, slot0 + step, ...: running (acc, M, z) per head for channel d.
-template <int G>
-__device__ __forceinline__ void finish_merge_range(const float *__restrict__ seg, int seg_stride, int slot0, int step,
-                                                   int count, float (*s_mz)[2 * G], float *acc, float *M, float *z, int d)
-{
-    constexpr int kB = (G == 8) ? 4 : 8;   // states whose loads are in flight together
-#pragma unroll
-    for (int o = 0; o < G; ++o) { acc[o] = 0.f; M[o] = neg_inf(); z[o] = 0.f; }
-    for (int base = 0; base < count; base += kB) {
-        float av[G][kB];
-#pragma unroll
-        for (int u = 0; u < kB; ++u) {
-            const bool on = base + u < count;
-            const float *sl = seg + (size_t)(slot0 + (on ? base + u : 0) * step) * seg_stride;
-#pragma unroll
-            for (int o = 0; o < G; ++o) av[o][u] = on ? ld_sync_f32(sl + o * kHeadDim + d) : 0.f;
-        }
-        float mz = 0.f;
-        const int u_mine = d / (2 * G), r_mine = d % (2 * G);   // (M, z) pairs of the batch: one word per thread
-        const bool mz_on = u_mine < kB && base + u_mine < count;
-        if (mz_on) mz = ld_sync_f32(seg + (size_t)(slot0 + (base + u_mine) * step) * seg_stride + G * kHeadDim + r_mine);
-        __syncthreads();                       // the previous batch's readers are done with s_mz
-        if (u_mine < kB) s_mz[u_mine][r_mine] = mz_on ? mz : (r_mine & 1 ? 0.f : neg_inf());
-        __syncthreads();
-#pragma unroll
-        for (int o = 0; o < G; ++o) {
-            float Mn = M[o];
-#pragma unroll
-            for (int u = 0; u < kB; ++u) Mn = fmaxf(Mn, s_mz[u][2 * o]);
-            const float Ms = (Mn == neg_inf()) ? 0.f : Mn;
-            const float keep = fast_exp2(M[o] - Ms);   // 0 while nothing has been merged yet
-            z[o] *= keep;
-            acc[o] *= keep;
-#pragma unroll
-            for (int u = 0; u < kB; ++u) {   // fixed order: deterministic
-                const float ew = fast_exp2(s_mz[u][2 * o] - Ms);
-                z[o] = fmaf(s_mz[u][2 * o + 1], ew, z[o]);
-                acc[o] = fmaf(av[o][u], ew, acc[o]);
-            }
-            M[o] = Mn;
-        }
-    }
-}
-
-template <int G>
-__global__ void __launch_bounds__(kFinThreads)
-finish_kernel(const int4 *__restrict__ piece_info, const unsigned long long *__restrict__ header,
-              unsigned long long *__restrict__ counters, float *__restrict__ seg, int seg_stride, int seg_slots,
-              float *__restrict__ o_part, float *__restrict__ m_part, float *__restrict__ lse_part, int n_units,
-              int Hkv, int Hq)
-{
-    static_assert(kFinThreads >= 8 * 2 * G, "one (M, z) word per thread and batch");
-    __shared__ float s_mz[8][2 * G];
-    __shared__ int s_last;
-    grid_dependency_wait();
-    grid_launch_dependents();
-    const int d = (int)threadIdx.x;
-    const int p = (int)blockIdx.x + 1;      // piece 0 cannot start inside a unit
-    const int n_pieces = (int)(ld_sync_u64(header + kHdrTotals) >> 32);
-    const int4 rec = ld_sync_int4(piece_info + min(p, kMaxSweepCtas + kMaxDynChunks - 1));
-    const unsigned long long epoch = ld_sync_u64(header + kHdrLastEpoch);
-    if (p >= n_pieces || rec.x < 0 || rec.w != (int)(unsigned)epoch) return;
-    const int unit = rec.x, first_slot = rec.y, nseg = rec.z;
-    if (unit >= n_units || nseg < 2 || first_slot < 0 || (long long)first_slot + nseg > (long long)seg_slots) return;
-    const int k = unit + p - first_slot;    // this piece's segment is the k-th of the unit
-    if (k < 1 || k >= nseg) return;
-    if (k != 1 && (k % kFinGroup) != 0) return;
-    const int group = k / kFinGroup, n_groups = (nseg + kFinGroup - 1) / kFinGroup;
-    const int seg0 = group * kFinGroup;
-    const size_t out_row = (size_t)(unit / Hkv) * Hq + (size_t)(unit % Hkv) * G;
-    const float kLn2 = 0.6931471805599453f;
-
-    float acc[G], M[G], z[G];
-    auto write_final = [&]() {
-#pragma unroll
-        for (int o = 0; o < G; ++o) {
-            const bool empty = (M[o] == neg_inf());
-            o_part[(out_row + o) * kHeadDim + d] = empty ? 0.f : acc[o] / z[o];
-            if (d == 0) {
-                m_part[out_row + o] = empty ? neg_inf() : M[o] * kLn2;
-                lse_part[out_row + o] = empty ? neg_inf() : (M[o] + log2f(z[o])) * kLn2;
-            }
-        }
-    };
-    finish_merge_range<G>(seg, seg_stride, first_slot + seg0, 1, min(kFinGroup, nseg - seg0), s_mz, acc, M, z, d);
-    if (n_groups == 1) { write_final(); return; }
-
-    // the group's partial state replaces the group's first segment (which only this CTA reads)
-    float *slot = seg + (size_t)(first_slot + seg0) * seg_stride;
-#pragma unroll
-    for (int o = 0; o < G; ++o) {
-        __stcg(slot + o * kHeadDim + d, acc[o]);
-        if (d == 0) { __stcg(slot + G * kHeadDim + 2 * o, M[o]); __stcg(slot + G * kHeadDim + 2 * o + 1, z[o]); }
-    }
-    __syncthreads();
-    if (d == 0) {
-        __threadfence();
-        s_last = (epoch_arrive(counters + unit, epoch) == (unsigned)n_groups) ? 1 : 0;
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    finish_merge_range<G>(seg, seg_stride, first_slot, kFinGroup, n_groups, s_mz, acc, M, z, d);
-    write_final();
-}
-
 // ------------------------------------------------------------------ bounded-wait self-test
 // Waits, with a short limit, on a barrier that nothing will ever complete, through the same wait
 // routine the sweep kernels use: the wait must give up, report QF_STATUS_TIMEOUT and let the kernel
@@ -868,7 +751,8 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
     *launches += 1;
     // one CTA per piece that can start inside a unit
     e = launch_pdl(finish_kernel<G>, dim3(n_ctas + kMaxDynChunks - 1), dim3(kFinThreads), 0, st,
-                   (const int4 *)piece_info, (const unsigned long long *)header, counters, seg, wsl.seg_stride,
+                   (const int4 *)piece_info, (const unsigned long long *)header, kMaxSweepCtas + kMaxDynChunks,
+                   counters, seg, wsl.seg_stride,
                    (int)wsl.seg_slots, o, m, l, n_entries * P.num_kv_heads, P.num_kv_heads, P.num_q_heads);
     if (e != cudaSuccess) { snprintf(msg, msg_len, "finish_kernel launch: %s", cudaGetErrorString(e)); return -5; }
     *launches += 1;
