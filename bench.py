@@ -285,8 +285,9 @@ def run_cuda(args):
             "e2e": {"value": whole_job_throughput(tot_bytes, e2e_ms / args.steps), "unit": "GB/s",
                     "h2d_bytes_per_step": hs.h2d_bytes, "d2h_bytes_per_step": hs.d2h_bytes,
                     "ms_per_step": e2e_ms / args.steps,
-                    "note": "qf_decode_step_host: q and step metadata copied in, out and lse copied back; "
-                            "the KV cache stays resident (only the query travels)"},
+                    "note": "qf_decode_step_host with pinned host buffers: a staging kernel reads q and the step "
+                            "metadata from host memory and the merge kernel writes out and lse to host memory "
+                            "(no copy-engine operations); the KV cache stays resident (only the query travels)"},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": {"bound": "hbm", "kernel": "sweep_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",

@@ -209,8 +209,14 @@ int qf_append_kv(void *k_cache, void *v_cache, const int32_t *block_table, const
  * the merge run, and the result is copied device -> host.  The KV cache stays
  * where it lives (that is the protocol: only the query travels).
  *
- *   host (pinned for true asynchrony): q_host, seq_lens_host,
- *       shard_ranges_host, shard_counts_host (may be NULL), out_host, lse_host
+ *   host: q_host, seq_lens_host, shard_ranges_host, shard_counts_host (may
+ *       be NULL), out_host, lse_host.  If all of them are page-locked and
+ *       mapped into the device's address space (cudaHostAlloc, or
+ *       cudaHostRegister with the mapped flag; out_host 16-byte aligned), no
+ *       copy operation is enqueued at all: one staging kernel reads the inputs
+ *       over the interconnect and the merge writes out/lse straight to the
+ *       host.  Any other host memory (pageable included) takes
+ *       cudaMemcpyAsync copies in and out; the results are the same bits.
  *   device: k_cache, v_cache, block_table (may be NULL), and `dev_scratch`
  *       of at least qf_step_scratch_bytes(p) bytes, 256-byte aligned, which
  *       holds the staged inputs, the shard states, the result and the sweep

@@ -2,6 +2,7 @@
 // carving and kernel launches.  See include/qf.h for the contract.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -239,6 +240,17 @@ int qf_append_kv(void *k_cache, void *v_cache, const int32_t *block_table, const
 
 // Carving of the step scratch used by qf_decode_step_host.
 namespace {
+// Device alias of a pinned, mapped host pointer; nullptr for any other kind of memory.
+void *mapped_alias(const void *host)
+{
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, host) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return (a.type == cudaMemoryTypeHost) ? a.devicePointer : nullptr;
+}
+
 struct StepLayout {
     size_t q, seq_lens, shard_ranges, shard_counts, o_part, m_part, lse_part, out, lse, workspace, total;
 };
@@ -283,15 +295,37 @@ int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_c
     char *base = (char *)dev_scratch;
     const size_t B = p->batch, S = p->max_shards, Hq = p->num_q_heads, D = p->head_dim;
     cudaError_t e;
-    e = cudaMemcpyAsync(base + L.q, q_host, B * Hq * D * 2, cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess) return cuda_fail(e, "copy q");
-    e = cudaMemcpyAsync(base + L.seq_lens, seq_lens_host, B * 4, cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess) return cuda_fail(e, "copy seq_lens");
-    e = cudaMemcpyAsync(base + L.shard_ranges, shard_ranges_host, B * S * 8, cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess) return cuda_fail(e, "copy shard_ranges");
-    if (shard_counts_host) {
-        e = cudaMemcpyAsync(base + L.shard_counts, shard_counts_host, B * 4, cudaMemcpyHostToDevice, st);
-        if (e != cudaSuccess) return cuda_fail(e, "copy shard_counts");
+    // Pinned, mapped host buffers are read and written by the kernels themselves: one staging launch
+    // instead of four copy operations in, and the merge writes the result straight to the host, so no
+    // copy operation out.  Any other kind of host memory takes the copy path.
+    const void *q_dev = mapped_alias(q_host), *sl_dev = mapped_alias(seq_lens_host);
+    const void *sr_dev = mapped_alias(shard_ranges_host);
+    const void *sc_dev = shard_counts_host ? mapped_alias(shard_counts_host) : nullptr;
+    float *out_dev = (float *)mapped_alias(out_host), *lse_dev = (float *)mapped_alias(lse_host);
+    const bool mapped = q_dev && sl_dev && sr_dev && (sc_dev || !shard_counts_host) && out_dev && lse_dev &&
+                        !((uintptr_t)out_dev & 15) && !((uintptr_t)q_dev & 3);
+    int extra_launches = 0;
+    if (mapped) {
+        const qf::IngestSpan sq = {(const uint32_t *)q_dev, (uint32_t *)(base + L.q), (unsigned)(B * Hq * D / 2)};
+        const qf::IngestSpan ssl = {(const uint32_t *)sl_dev, (uint32_t *)(base + L.seq_lens), (unsigned)B};
+        const qf::IngestSpan ssr = {(const uint32_t *)sr_dev, (uint32_t *)(base + L.shard_ranges), (unsigned)(B * S * 2)};
+        const qf::IngestSpan ssc = {(const uint32_t *)sc_dev, (uint32_t *)(base + L.shard_counts),
+                                    shard_counts_host ? (unsigned)B : 0u};
+        const unsigned blocks = (unsigned)std::min<size_t>(148, (B * Hq * D / 8 + 255) / 256 + 1);
+        e = qf::launch_pdl(qf::ingest_kernel, dim3(blocks), dim3(256), 0, st, sq, ssl, ssr, ssc);
+        if (e != cudaSuccess) return cuda_fail(e, "ingest_kernel launch");
+        extra_launches = 1;
+    } else {
+        e = cudaMemcpyAsync(base + L.q, q_host, B * Hq * D * 2, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return cuda_fail(e, "copy q");
+        e = cudaMemcpyAsync(base + L.seq_lens, seq_lens_host, B * 4, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return cuda_fail(e, "copy seq_lens");
+        e = cudaMemcpyAsync(base + L.shard_ranges, shard_ranges_host, B * S * 8, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return cuda_fail(e, "copy shard_ranges");
+        if (shard_counts_host) {
+            e = cudaMemcpyAsync(base + L.shard_counts, shard_counts_host, B * 4, cudaMemcpyHostToDevice, st);
+            if (e != cudaSuccess) return cuda_fail(e, "copy shard_counts");
+        }
     }
     rc = qf_decode_partial(base + L.q, k_cache, v_cache, block_table, (const int32_t *)(base + L.seq_lens),
                            (const int32_t *)(base + L.shard_ranges), (float *)(base + L.o_part),
@@ -301,13 +335,16 @@ int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_c
     const int sweep_launches = g_last_launches;
     rc = qf_combine((const float *)(base + L.o_part), (const float *)(base + L.lse_part),
                     shard_counts_host ? (const int32_t *)(base + L.shard_counts) : nullptr,
-                    (float *)(base + L.out), (float *)(base + L.lse), p, cuda_stream);
+                    mapped ? out_dev : (float *)(base + L.out), mapped ? lse_dev : (float *)(base + L.lse), p,
+                    cuda_stream);
     if (rc != QF_OK) return rc;
-    g_last_launches += sweep_launches;
-    e = cudaMemcpyAsync(out_host, base + L.out, B * Hq * D * 4, cudaMemcpyDeviceToHost, st);
-    if (e != cudaSuccess) return cuda_fail(e, "copy out");
-    e = cudaMemcpyAsync(lse_host, base + L.lse, B * Hq * 4, cudaMemcpyDeviceToHost, st);
-    if (e != cudaSuccess) return cuda_fail(e, "copy lse");
+    g_last_launches += sweep_launches + extra_launches;
+    if (!mapped) {
+        e = cudaMemcpyAsync(out_host, base + L.out, B * Hq * D * 4, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return cuda_fail(e, "copy out");
+        e = cudaMemcpyAsync(lse_host, base + L.lse, B * Hq * 4, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return cuda_fail(e, "copy lse");
+    }
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
     return QF_OK;

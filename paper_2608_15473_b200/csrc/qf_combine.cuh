@@ -148,4 +148,31 @@ append_kv_kernel(uint16_t *__restrict__ k_cache, uint16_t *__restrict__ v_cache,
     *reinterpret_cast<uint2 *>(v_cache + dst) = *reinterpret_cast<const uint2 *>(v_new + src);
 }
 
+// Staging of a decode step's inputs from pinned, mapped host memory: the kernel reads the host buffers
+// over the interconnect itself (four spans, one launch) instead of four copy-engine operations.
+// Spans are sequences of 32-bit words; `words16` of them, from the start, move as 16-byte words.
+struct IngestSpan {
+    const uint32_t *src;   // device alias of the host buffer
+    uint32_t *dst;
+    unsigned words;        // 32-bit words
+};
+__global__ void __launch_bounds__(256)
+ingest_kernel(IngestSpan a, IngestSpan b, IngestSpan c, IngestSpan d)
+{
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const unsigned tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    const IngestSpan spans[4] = {a, b, c, d};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const IngestSpan sp = spans[k];
+        if (sp.words == 0) continue;
+        const bool wide = (((uintptr_t)sp.src | (uintptr_t)sp.dst) & 15) == 0;
+        const unsigned n16 = wide ? sp.words / 4 : 0;
+        for (unsigned i = tid; i < n16; i += nth)
+            reinterpret_cast<uint4 *>(sp.dst)[i] = reinterpret_cast<const uint4 *>(sp.src)[i];
+        for (unsigned i = n16 * 4 + tid; i < sp.words; i += nth) sp.dst[i] = sp.src[i];
+    }
+}
+
 }  // namespace qf

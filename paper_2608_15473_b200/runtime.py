@@ -84,15 +84,18 @@ class DeviceWorkload:
 class HostStepper:
     """End-to-end stepping from pinned host buffers through qf_decode_step_host."""
 
-    def __init__(self, dw: DeviceWorkload):
+    def __init__(self, dw: DeviceWorkload, pinned: bool = True):
+        """pinned=True: page-locked (and therefore mapped) host buffers, which the library's kernels read and
+        write directly; pinned=False: ordinary pageable buffers, which take the library's copy path."""
         self.dw = dw
         w = dw.w
-        self.q_host = torch.from_numpy(w.q.view(np.int16).copy()).pin_memory()
-        self.seq_lens_host = torch.from_numpy(w.seq_lens.copy()).pin_memory()
-        self.shard_ranges_host = torch.from_numpy(w.shard_ranges.copy()).pin_memory()
-        self.shard_counts_host = torch.from_numpy(w.shard_counts.copy()).pin_memory()
-        self.out_host = torch.empty((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32).pin_memory()
-        self.lse_host = torch.empty((w.batch, w.num_q_heads), dtype=torch.float32).pin_memory()
+        pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+        self.q_host = pin(torch.from_numpy(w.q.view(np.int16).copy()))
+        self.seq_lens_host = pin(torch.from_numpy(w.seq_lens.copy()))
+        self.shard_ranges_host = pin(torch.from_numpy(w.shard_ranges.copy()))
+        self.shard_counts_host = pin(torch.from_numpy(w.shard_counts.copy()))
+        self.out_host = pin(torch.empty((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32))
+        self.lse_host = pin(torch.empty((w.batch, w.num_q_heads), dtype=torch.float32))
         self.scratch_bytes = qf.step_scratch_bytes(dw.params)
         self.scratch = torch.empty(self.scratch_bytes, dtype=torch.uint8, device=dw.device)
         self.h2d_bytes = (self.q_host.numel() * 2 + self.seq_lens_host.numel() * 4 +

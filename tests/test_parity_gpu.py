@@ -331,15 +331,32 @@ def test_bad_page_index_is_reported_not_followed(flags):
     assert T.out_err(got[3][1], ref[3][1]) < T.ENG_OUT and T.lse_err(got[4][1], ref[4][1]) < T.ENG_LSE
 
 
-def test_host_step_matches_device_path():
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_step_matches_device_path(pinned):
+    # pinned host buffers are read and written by the kernels themselves (one staging launch more, no copy
+    # operations); pageable ones go through copies: the same bits either way
     w = wl.config3(seed=7, batch=5, hi=6000)
     dw = run(w)
-    hs = HostStepper(dw)
+    device_launches = dw.step()
+    hs = HostStepper(dw, pinned=pinned)
+    hs.out_host.fill_(float("nan"))
+    hs.lse_host.fill_(float("nan"))
     hs.step()
+    assert qf.last_launch_count() == device_launches + (1 if pinned else 0)
     _, _, _, out, lse = dw.results()
     assert np.array_equal(hs.out_host.numpy().astype(np.float64), out)
     assert np.array_equal(hs.lse_host.numpy().astype(np.float64), lse)
     assert hs.h2d_bytes > 0 and hs.d2h_bytes == out.size * 4 + lse.size * 4
+    # a second step with a new query through the same buffers
+    rng = np.random.default_rng(5)
+    w.q = wl.f32_to_bf16_bits(rng.standard_normal(w.q.shape).astype(np.float32))
+    hs.q_host.copy_(torch.from_numpy(w.q.view(np.int16)))
+    hs.step()
+    dw.q.copy_(torch.from_numpy(w.q.view(np.int16)).view(torch.bfloat16).cuda())
+    dw.step()
+    _, _, _, out, lse = dw.results()
+    assert np.array_equal(hs.out_host.numpy().astype(np.float64), out)
+    assert np.array_equal(hs.lse_host.numpy().astype(np.float64), lse)
 
 
 # T8: the benchmark configurations at full size, sampled outputs
