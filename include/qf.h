@@ -250,6 +250,21 @@ int qf_read_status(const void *workspace, int32_t *host_status, void *cuda_strea
 int qf_selftest_bounded_wait(void *workspace, void *cuda_stream);
 
 /*
+ * Diagnostic aid (no counterpart in the paper; host only, no GPU needed).  The
+ * sweep cuts its work, `total_units` stage units of 128 tokens of one KV head,
+ * into pieces: one static slice per CTA, then, for sweeps long enough (or any
+ * sweep of at least two units per CTA with draw_always != 0), chunks of
+ * halving size that CTAs draw from a counter.  This returns the number of
+ * pieces the kernels would use for (total_units, n_ctas) and writes the first
+ * min(pieces, capacity) ranges [piece_begin[p], piece_end[p]); it also checks
+ * that the kernels' position-to-piece map agrees with the ranges.  Negative
+ * return: QF_ERR_BAD_SHAPE (arguments out of range, or the two maps disagree),
+ * QF_ERR_NULL.  n_ctas is at most 160.
+ */
+int qf_plan_pieces(int total_units, int n_ctas, int draw_always, int32_t *piece_begin,
+                   int32_t *piece_end, int capacity);
+
+/*
  * Number of kernels the last qf_decode_partial / qf_combine call on this
  * thread enqueued (for launch accounting in benchmarks).
  */

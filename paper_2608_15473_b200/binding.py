@@ -38,7 +38,7 @@ EXPORTS = (
     "qf_version", "qf_strerror", "qf_workspace_bytes", "qf_decode_partial", "qf_combine",
     "qf_step_scratch_bytes", "qf_decode_step_host", "qf_read_status", "qf_last_launch_count",
     "qf_set_profile_events", "qf_decode_partial_static", "qf_static_scratch_error",
-    "qf_combine_self", "qf_append_kv", "qf_selftest_bounded_wait",
+    "qf_combine_self", "qf_append_kv", "qf_selftest_bounded_wait", "qf_plan_pieces",
 )
 
 
@@ -105,6 +105,8 @@ def lib() -> ctypes.CDLL:
         L.qf_decode_partial_static.restype = ctypes.c_int
         L.qf_decode_partial_static.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, vp, vp, pp, vp]
         L.qf_static_scratch_error.restype = ctypes.c_char_p
+        L.qf_plan_pieces.restype = ctypes.c_int
+        L.qf_plan_pieces.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, i32p, i32p, ctypes.c_int]
         _lib = L
     return _lib
 
@@ -229,6 +231,18 @@ def selftest_bounded_wait(workspace, stream=None) -> None:
     rc = lib().qf_selftest_bounded_wait(_ptr(workspace), _stream(stream))
     if rc != QF_OK:
         raise QFError(rc, "qf_selftest_bounded_wait")
+
+
+def plan_pieces(total_units: int, n_ctas: int, draw_always: bool = False):
+    """The sweep's schedule for (total_units, n_ctas): a list of [begin, end) ranges, one per piece
+    (static slices first, then the drawn chunks).  Host arithmetic only: no GPU is touched."""
+    cap = n_ctas + 4096
+    b = (ctypes.c_int32 * cap)()
+    e = (ctypes.c_int32 * cap)()
+    n = lib().qf_plan_pieces(int(total_units), int(n_ctas), int(bool(draw_always)), b, e, cap)
+    if n < 0:
+        raise QFError(n, "qf_plan_pieces")
+    return [(int(b[i]), int(e[i])) for i in range(n)]
 
 
 def read_status(workspace, stream=None) -> int:

@@ -350,6 +350,26 @@ int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_c
     return QF_OK;
 }
 
+int qf_plan_pieces(int total_units, int n_ctas, int draw_always, int32_t *piece_begin, int32_t *piece_end,
+                   int capacity)
+{
+    if (total_units < 0 || n_ctas < 1 || n_ctas > qf::kMaxSweepCtas || capacity < 0) return QF_ERR_BAD_SHAPE;
+    if (capacity > 0 && (!piece_begin || !piece_end)) return QF_ERR_NULL;
+    const qf::PieceGrid g = qf::piece_grid(total_units, n_ctas, true, draw_always != 0);
+    const int n = n_ctas + g.n_chunks;
+    for (int p = 0; p < n && p < capacity; ++p) {
+        int b, e;
+        qf::piece_range(g, n_ctas, p, b, e);
+        piece_begin[p] = b;
+        piece_end[p] = e;
+        // the inverse map the kernels use must agree with the ranges
+        for (int x = b; x < e; x += (e - b > 64 ? (e - b) / 7 + 1 : 1))
+            if (qf::piece_of(g, n_ctas, x) != p) return QF_ERR_BAD_SHAPE;
+        if (e > b && qf::piece_of(g, n_ctas, e - 1) != p) return QF_ERR_BAD_SHAPE;
+    }
+    return n;
+}
+
 int qf_selftest_bounded_wait(void *workspace, void *cuda_stream)
 {
     if (!workspace) return QF_ERR_NULL;

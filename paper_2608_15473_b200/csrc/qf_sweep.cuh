@@ -124,12 +124,14 @@ struct PieceGrid {
     int r_first[kDynRounds + 1];   // first chunk of round r
     int r_size[kDynRounds];        // units per chunk in round r (the round's last chunk may be shorter)
 };
-__device__ __forceinline__ PieceGrid piece_grid(int total, int n_ctas, bool allow_dynamic, bool always)
+__host__ __device__ __forceinline__ int imin(int a, int b) { return a < b ? a : b; }
+__host__ __device__ __forceinline__ int imax(int a, int b) { return a > b ? a : b; }
+__host__ __device__ __forceinline__ PieceGrid piece_grid(int total, int n_ctas, bool allow_dynamic, bool always)
 {
     PieceGrid g;
     const int min_total = always ? 2 * n_ctas : n_ctas * kDynMinUnitsPerCta;   // static slices of at least one unit
     if (!allow_dynamic || total < min_total) {
-        g.slice = max(1, (total + n_ctas - 1) / n_ctas);
+        g.slice = imax(1, (total + n_ctas - 1) / n_ctas);
         g.static_end = total;
     } else {
         g.slice = (total - total / kDynDivisor) / n_ctas;
@@ -140,7 +142,7 @@ __device__ __forceinline__ PieceGrid piece_grid(int total, int n_ctas, bool allo
     for (int r = 0; r < kDynRounds; ++r) {
         const int rem = total - off;
         const int share = (r == kDynRounds - 1) ? rem : (rem + 1) / 2;
-        const int size = max(kDynMinChunk, (share + n_ctas - 1) / n_ctas);
+        const int size = imax(kDynMinChunk, (share + n_ctas - 1) / n_ctas);
         g.r_start[r] = off;
         g.r_first[r] = idx;
         g.r_size[r] = size;
@@ -152,7 +154,7 @@ __device__ __forceinline__ PieceGrid piece_grid(int total, int n_ctas, bool allo
     g.n_chunks = idx;
     return g;
 }
-__device__ __forceinline__ int piece_of(const PieceGrid &g, int n_ctas, int pos)
+__host__ __device__ __forceinline__ int piece_of(const PieceGrid &g, int n_ctas, int pos)
 {
     if (pos < g.static_end) return pos / g.slice;
     int piece = 0;
@@ -161,11 +163,12 @@ __device__ __forceinline__ int piece_of(const PieceGrid &g, int n_ctas, int pos)
         if (pos >= g.r_start[r] && pos < g.r_start[r + 1]) piece = n_ctas + g.r_first[r] + (pos - g.r_start[r]) / g.r_size[r];
     return piece;
 }
-__device__ __forceinline__ void piece_range(const PieceGrid &g, int n_ctas, int piece, int &pos0, int &pos1)
+__host__ __device__ __forceinline__ void piece_range(const PieceGrid &g, int n_ctas, int piece, int &pos0, int &pos1)
 {
     if (piece < n_ctas) {
-        pos0 = (int)min((long long)g.static_end, (long long)piece * g.slice);
-        pos1 = (int)min((long long)g.static_end, (long long)(piece + 1) * g.slice);
+        const long long lo = (long long)piece * g.slice, hi = lo + g.slice;
+        pos0 = lo < g.static_end ? (int)lo : g.static_end;
+        pos1 = hi < g.static_end ? (int)hi : g.static_end;
         return;
     }
     const int k = piece - n_ctas;
@@ -174,7 +177,7 @@ __device__ __forceinline__ void piece_range(const PieceGrid &g, int n_ctas, int 
     for (int r = 0; r < kDynRounds; ++r)
         if (k >= g.r_first[r] && k < g.r_first[r + 1]) {
             pos0 = g.r_start[r] + (k - g.r_first[r]) * g.r_size[r];
-            pos1 = min(pos0 + g.r_size[r], g.r_start[r + 1]);
+            pos1 = imin(pos0 + g.r_size[r], g.r_start[r + 1]);
         }
 }
 
