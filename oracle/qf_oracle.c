@@ -17,7 +17,11 @@
  * sharded == unsharded, pairwise fold == n-way merge, overflow cases at
  * log Z = 100, shift invariance, d(out)/d(v_j) = A_j, paging invariance,
  * SciPy / PyTorch fp64 library routines, exact-rational brute force on tiny
- * inputs.  Nothing here is "parity unpinned".
+ * inputs.  The projection pair at the end of the file (u' = z + W_o a,
+ * q = W_q N_1(u')) has its own pins: one-hot inputs that read out weight
+ * columns, exact row sums under a constant stream, power-of-two equivariance,
+ * PyTorch fp64 matmul and rms_norm, exact rational brute force, nearest-bf16
+ * checks of every rounding.  Nothing here is "parity unpinned".
  *
  * Conventions where the paper is silent (stated again in the design notes):
  *   - q, K, V are bf16 bit patterns, widened exactly to fp64.
@@ -383,3 +387,86 @@ int qfo_self_fold(const double *o_prev, const double *lse_prev, const uint16_t *
     return 0;
 }
 
+
+/* ------------------------------------------------------------------------
+ * The cache side's projection pair at a layer boundary (Section 4 "what each
+ * side holds": W_q and W_o live with the cache; the stage's contract ends in
+ * u' = z + W_o a, and the next stage opens with q = W_q N_1(u'); the appendix
+ * "The cache side must batch" makes it a product over the co-resident
+ * requests of a batch).
+ *
+ * The paper fixes bf16 weights and a bf16 residual stream (its per-layer byte
+ * counts) and leaves the rest open; the reading taken here, stated again in
+ * the design notes:
+ *   - a  [M][n_q]      fp32, the attention output of the layer (what the merge
+ *                      returns), rounded to bf16 before the product;
+ *   - z  [M][d_model]  bf16, the residual stream after the feed-forward;
+ *   - w_o [d_model][n_q], w_q [n_q][d_model], g [d_model]  bf16;
+ *   - N_1 is the root-mean-square normalisation with gain g:
+ *         N_1(u)_i = g_i u_i / sqrt(mean_j u_j^2 + eps);
+ *   - u' is rounded to bf16 (it is the stream that goes on the wire) and the
+ *     normalisation reads the rounded stream; x = N_1(u') is rounded to bf16
+ *     (it is the operand of the second product); q is rounded to bf16 (it is
+ *     what the sweep consumes).
+ * Every rounding is value -> nearest binary32 -> nearest bf16, ties to even,
+ * the two steps a kernel with an fp32 accumulator takes; the sums themselves
+ * are exact products of bf16 values accumulated in fp64.
+ *   u_out [M][d_model], q_out [M][n_q]   bf16 bit patterns
+ *   u_exact, q_exact (optional, fp64)    the values before their last rounding
+ * ------------------------------------------------------------------------ */
+static uint16_t f64_to_bf16_via_f32(double x)
+{
+    float f = (float)x; /* round to nearest even (default rounding mode) */
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40u); /* NaN stays NaN */
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+int qfo_project_pair(int32_t M, int32_t d_model, int32_t n_q, const float *a, const uint16_t *z,
+                     const uint16_t *w_o, const uint16_t *g, double eps, const uint16_t *w_q,
+                     uint16_t *u_out, uint16_t *q_out, double *u_exact, double *q_exact)
+{
+    if (M <= 0 || d_model <= 0 || n_q <= 0) return -1;
+    double *ab = (double *)malloc(sizeof(double) * (size_t)M * (size_t)n_q);
+    double *x = (double *)malloc(sizeof(double) * (size_t)M * (size_t)d_model);
+    if (!ab || !x) { free(ab); free(x); return -2; }
+    for (int64_t i = 0; i < (int64_t)M * n_q; ++i) ab[i] = bf16_to_f64(f64_to_bf16_via_f32((double)a[i]));
+
+    /* u' = z + W_o a */
+#pragma omp parallel for schedule(static)
+    for (int64_t idx = 0; idx < (int64_t)M * d_model; ++idx) {
+        const int64_t m = idx / d_model, o = idx % d_model;
+        double acc = 0.0;
+        for (int k = 0; k < n_q; ++k) acc += bf16_to_f64(w_o[o * (int64_t)n_q + k]) * ab[m * (int64_t)n_q + k];
+        const double u = bf16_to_f64(z[idx]) + acc;
+        if (u_exact) u_exact[idx] = u;
+        u_out[idx] = f64_to_bf16_via_f32(u);
+    }
+    /* x = N_1(u') on the rounded stream */
+    for (int m = 0; m < M; ++m) {
+        double ss = 0.0;
+        for (int i = 0; i < d_model; ++i) {
+            const double u = bf16_to_f64(u_out[(int64_t)m * d_model + i]);
+            ss += u * u;
+        }
+        const double rstd = 1.0 / sqrt(ss / (double)d_model + eps);
+        for (int i = 0; i < d_model; ++i) {
+            const double u = bf16_to_f64(u_out[(int64_t)m * d_model + i]);
+            x[(int64_t)m * d_model + i] = bf16_to_f64(f64_to_bf16_via_f32(bf16_to_f64(g[i]) * u * rstd));
+        }
+    }
+    /* q = W_q x */
+#pragma omp parallel for schedule(static)
+    for (int64_t idx = 0; idx < (int64_t)M * n_q; ++idx) {
+        const int64_t m = idx / n_q, o = idx % n_q;
+        double acc = 0.0;
+        for (int k = 0; k < d_model; ++k) acc += bf16_to_f64(w_q[o * (int64_t)d_model + k]) * x[m * (int64_t)d_model + k];
+        if (q_exact) q_exact[idx] = acc;
+        q_out[idx] = f64_to_bf16_via_f32(acc);
+    }
+    free(ab);
+    free(x);
+    return 0;
+}

@@ -213,3 +213,28 @@ def self_fold(o_prev, lse_prev, q, k_new, v_new, sh: Shape):
     assert rc == 0
     return out, lse, s_self
 
+
+
+def project_pair(a, z, w_o, g, w_q, eps=1e-6, exact=False):
+    """The cache side's projection pair (Section 4; appendix "The cache side must batch"):
+    u' = z + W_o a, q = W_q N_1(u') with bf16 roundings of a, u', N_1(u') and q.
+    a: float32 [M, n_q]; z: bf16 bits [M, d_model]; w_o: [d_model, n_q]; g: [d_model]; w_q: [n_q, d_model].
+    Returns (u bf16 bits, q bf16 bits) and, with exact=True, the fp64 values before the last rounding."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    z, w_o, g, w_q = (np.ascontiguousarray(t, dtype=np.uint16) for t in (z, w_o, g, w_q))
+    M, n_q = a.shape
+    d_model = z.shape[1]
+    assert z.shape == (M, d_model) and w_o.shape == (d_model, n_q) and w_q.shape == (n_q, d_model) and g.shape == (d_model,)
+    u = np.empty((M, d_model), np.uint16)
+    q = np.empty((M, n_q), np.uint16)
+    ue = np.empty((M, d_model), np.float64) if exact else None
+    qe = np.empty((M, n_q), np.float64) if exact else None
+    f = lib().qfo_project_pair
+    f.restype = ctypes.c_int
+    vp = ctypes.c_void_p
+    f.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp, vp, ctypes.c_double, vp, vp, vp, vp, vp]
+    rc = f(M, d_model, n_q, a.ctypes.data, z.ctypes.data, w_o.ctypes.data, g.ctypes.data, float(eps), w_q.ctypes.data,
+           u.ctypes.data, q.ctypes.data, ue.ctypes.data if exact else None, qe.ctypes.data if exact else None)
+    if rc != 0:
+        raise RuntimeError(f"qfo_project_pair failed: {rc}")
+    return (u, q, ue, qe) if exact else (u, q)
