@@ -204,6 +204,40 @@ int qf_append_kv(void *k_cache, void *v_cache, const int32_t *block_table, const
                  const qf_params *p, void *cuda_stream);
 
 /*
+ * Section 4 ("what each side holds": W_q and W_o live with the cache) and the
+ * appendix paragraph "The cache side must batch": the projection pair at a
+ * layer boundary, over the co-resident requests of a batch,
+ *     u' = z + W_o a              (closes the layer:  [batch, d_model])
+ *     q  = W_q N_1(u')            (opens the next:    [batch, n_q])
+ * with N_1 the root-mean-square normalisation with gain g,
+ *     N_1(u)_i = g_i u_i / sqrt(mean_j u_j^2 + eps).
+ * The paper fixes bf16 weights and a bf16 stream; the rest is this library's
+ * reading: a is the fp32 attention output (what qf_combine / qf_combine_self
+ * return, [batch, n_q] = [batch, Hq, D]) and is rounded to bf16 before the
+ * product; products accumulate in fp32; u' is rounded to bf16 and N_1 reads
+ * the rounded stream; N_1(u') and q are rounded to bf16.  q has the layout
+ * qf_decode_partial consumes.
+ *   a [batch, n_q] fp32; z, u_out [batch, d_model] bf16; w_o [d_model, n_q],
+ *   w_q [n_q, d_model], g [d_model] bf16, row-major; q_out [batch, n_q] bf16.
+ *   All device pointers; a, z, g, u_out, q_out 16-byte aligned, the weights
+ *   128-byte aligned.  workspace: qf_project_workspace_bytes bytes, 256-byte
+ *   aligned, contents need not be initialised.
+ * Supported: 1 <= batch <= 64; d_model and n_q multiples of 512, at most
+ * 5,120 (for batch > 32: at least 1,024 and at most 4,096, which the
+ * shared-memory budget sets); else
+ * QF_ERR_UNSUPPORTED (qf_project_workspace_bytes returns 0).  Larger batches
+ * are run in slices of 64 by the caller.  Enqueues two kernels on cuda_stream.
+ * qf_project_status copies the pair's status word (QF_STATUS_TIMEOUT if a
+ * bounded wait inside a kernel ran out; 0 = clean) and synchronises the stream.
+ */
+size_t qf_project_workspace_bytes(int batch, int d_model, int n_q);
+int qf_project_pair(const float *a, const void *z, const void *w_o, const void *g,
+                    const void *w_q, void *u_out, void *q_out,
+                    int batch, int d_model, int n_q, float eps,
+                    void *workspace, size_t workspace_bytes, void *cuda_stream);
+int qf_project_status(const void *workspace, int32_t *host_status, void *cuda_stream);
+
+/*
  * One whole decode step driven from HOST buffers, as a serving loop calls it:
  * the query and the step's metadata are copied host -> device, the sweep and
  * the merge run, and the result is copied device -> host.  The KV cache stays

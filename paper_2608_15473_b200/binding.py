@@ -39,6 +39,7 @@ EXPORTS = (
     "qf_step_scratch_bytes", "qf_decode_step_host", "qf_read_status", "qf_last_launch_count",
     "qf_set_profile_events", "qf_decode_partial_static", "qf_static_scratch_error",
     "qf_combine_self", "qf_append_kv", "qf_selftest_bounded_wait", "qf_plan_pieces",
+    "qf_project_workspace_bytes", "qf_project_pair", "qf_project_status",
 )
 
 
@@ -105,6 +106,13 @@ def lib() -> ctypes.CDLL:
         L.qf_decode_partial_static.restype = ctypes.c_int
         L.qf_decode_partial_static.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, vp, vp, pp, vp]
         L.qf_static_scratch_error.restype = ctypes.c_char_p
+        L.qf_project_workspace_bytes.restype = ctypes.c_size_t
+        L.qf_project_workspace_bytes.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int]
+        L.qf_project_pair.restype = ctypes.c_int
+        L.qf_project_pair.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                      ctypes.c_float, vp, ctypes.c_size_t, vp]
+        L.qf_project_status.restype = ctypes.c_int
+        L.qf_project_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
         L.qf_plan_pieces.restype = ctypes.c_int
         L.qf_plan_pieces.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, i32p, i32p, ctypes.c_int]
         _lib = L
@@ -231,6 +239,30 @@ def selftest_bounded_wait(workspace, stream=None) -> None:
     rc = lib().qf_selftest_bounded_wait(_ptr(workspace), _stream(stream))
     if rc != QF_OK:
         raise QFError(rc, "qf_selftest_bounded_wait")
+
+
+def project_workspace_bytes(batch: int, d_model: int, n_q: int) -> int:
+    return int(lib().qf_project_workspace_bytes(int(batch), int(d_model), int(n_q)))
+
+
+def project_pair(a, z, w_o, g, w_q, u_out, q_out, eps, workspace, stream=None, check=True) -> int:
+    """u' = z + W_o a, q = W_q N_1(u') for a batch of co-resident requests (device tensors; marshalling only)."""
+    batch, n_q = int(a.shape[0]), int(a.shape[1])
+    d_model = int(z.shape[1])
+    rc = lib().qf_project_pair(_ptr(a), _ptr(z), _ptr(w_o), _ptr(g), _ptr(w_q), _ptr(u_out), _ptr(q_out), batch,
+                               d_model, n_q, float(eps), _ptr(workspace),
+                               int(workspace.numel() * workspace.element_size()), _stream(stream))
+    if check and rc != QF_OK:
+        raise QFError(rc, "qf_project_pair")
+    return rc
+
+
+def project_status(workspace, stream=None) -> int:
+    st = ctypes.c_int32(0)
+    rc = lib().qf_project_status(_ptr(workspace), ctypes.byref(st), _stream(stream))
+    if rc != QF_OK:
+        raise QFError(rc, "qf_project_status")
+    return int(st.value)
 
 
 def plan_pieces(total_units: int, n_ctas: int, draw_always: bool = False):

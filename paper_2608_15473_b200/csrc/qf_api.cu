@@ -10,6 +10,7 @@
 #include "../../include/qf.h"
 #include "qf_combine.cuh"
 #include "qf_common.cuh"
+#include "qf_proj.cuh"
 #include "qf_simple.cuh"
 #include "qf_sweep.cuh"
 
@@ -347,6 +348,63 @@ int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_c
     }
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    return QF_OK;
+}
+
+size_t qf_project_workspace_bytes(int batch, int d_model, int n_q)
+{
+    if (!qf::proj_shape_ok(batch, d_model, n_q) || !qf::proj_shape_ok(batch, n_q, d_model)) return 0;
+    // a status word, then one row of per-request sums of squares per 128-feature tile of the stream
+    return align256(256 + (size_t)(d_model / qf::kProjTileOut) * qf::kProjMaxBatch * sizeof(float));
+}
+
+int qf_project_pair(const float *a, const void *z, const void *w_o, const void *g, const void *w_q, void *u_out,
+                    void *q_out, int batch, int d_model, int n_q, float eps, void *workspace, size_t workspace_bytes,
+                    void *cuda_stream)
+{
+    g_last_launches = 0;
+    if (batch < 1 || d_model < 1 || n_q < 1 || !(eps >= 0.f)) return QF_ERR_BAD_SHAPE;
+    if (!qf::proj_shape_ok(batch, d_model, n_q) || !qf::proj_shape_ok(batch, n_q, d_model)) return QF_ERR_UNSUPPORTED;
+    if (!a || !z || !w_o || !g || !w_q || !u_out || !q_out) return QF_ERR_NULL;
+    if (((uintptr_t)a & 15) || ((uintptr_t)z & 15) || ((uintptr_t)g & 15) || ((uintptr_t)u_out & 15) ||
+        ((uintptr_t)q_out & 15) || ((uintptr_t)w_o & 127) || ((uintptr_t)w_q & 127))
+        return QF_ERR_BAD_SHAPE;
+    const size_t need = qf_project_workspace_bytes(batch, d_model, n_q);
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return QF_ERR_WORKSPACE;
+    int rc = check_device(nullptr);
+    if (rc != QF_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    CUtensorMap map_o, map_q;
+    if (qf::make_weight_map(&map_o, w_o, d_model, n_q, g_cuda_msg, sizeof g_cuda_msg)) return QF_ERR_CUDA;
+    if (qf::make_weight_map(&map_q, w_q, n_q, d_model, g_cuda_msg, sizeof g_cuda_msg)) return QF_ERR_CUDA;
+    unsigned *status = (unsigned *)workspace;
+    float *ssq_part = (float *)((char *)workspace + 256);
+
+    qf::ProjArgs s0 = {};
+    s0.a = a; s0.z = (const uint16_t *)z; s0.out = (uint16_t *)u_out; s0.ssq_part = ssq_part; s0.status = status;
+    s0.batch = batch; s0.n_out = d_model; s0.k_total = n_q;
+    cudaError_t e = qf::launch_proj<0>(map_o, s0, st);
+    if (e != cudaSuccess) return cuda_fail(e, "proj_kernel<0> launch");
+    qf::ProjArgs s1 = {};
+    s1.u_in = (const uint16_t *)u_out; s1.g = (const uint16_t *)g; s1.out = (uint16_t *)q_out; s1.ssq_part = ssq_part;
+    s1.status = status; s1.batch = batch; s1.n_out = n_q; s1.k_total = d_model;
+    s1.ssq_tiles = d_model / qf::kProjTileOut; s1.inv_d_model = 1.0f / (float)d_model; s1.eps = eps;
+    e = qf::launch_proj<1>(map_q, s1, st);
+    if (e != cudaSuccess) return cuda_fail(e, "proj_kernel<1> launch");
+    g_last_launches = 2;
+    return QF_OK;
+}
+
+int qf_project_status(const void *workspace, int32_t *host_status, void *cuda_stream)
+{
+    if (!workspace || !host_status) return QF_ERR_NULL;
+    unsigned word = 0;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMemcpyAsync(&word, workspace, sizeof word, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync");
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    *host_status = (int32_t)word;
     return QF_OK;
 }
 

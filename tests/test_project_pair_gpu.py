@@ -1,0 +1,157 @@
+"""GPU parity of the cache side's projection pair (u' = z + W_o a, q = W_q N_1(u')) against the fp64 oracle.
+
+Tolerance.  Both sides round value -> binary32 -> bf16 at the same three points, so most outputs are the same
+bits.  The kernel's sums carry fp32 accumulation error, a few 1e-7 of the row's scale, which shows in two
+ways: (1) now and then it carries a value across a bf16 rounding boundary, and the output differs by one
+bf16 unit in the last place of the value; (2) where the sum nearly cancels, the value is so small that the
+same absolute error is several of ITS units in the last place.  A u' element that flipped (one part in 2^8
+of it; about one element in 4,000 does) changes that request's normalised operand x_k by the same share, and
+through it every q of the request by |W_q[o,k]| 2^-8 |x_k|: with |W_q| up to about 4/sqrt(d_model) and |x_k|
+up to about 4 that is up to 1e-3 of the row's scale, and a row may hold two flips.  So an element passes if
+    |got - ref| <= ulp_bf16(max(|got|, |ref|)) + abs_tol * rms(row),   abs_tol = 1e-5 for u', 2.5e-3 for q
+(for q that is two thirds of a bf16 unit in the last place of a typical element), and the share of elements
+that differ at all is bounded (1 % for u', 5 % for q; measured 0.03 % and 0.2-1.6 %)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import qf_oracle as orc
+from paper_2608_15473_b200 import binding as qf
+from paper_2608_15473_b200 import build as qf_build
+from paper_2608_15473_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    qf_build.build()
+
+
+def bits_to_f64(b):
+    return (np.asarray(b, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def dev_bf16(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).cuda()
+
+
+def host_bits(t):
+    return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def make_inputs(batch, d_model, n_q, seed):
+    rng = np.random.default_rng(seed)
+    sc_o, sc_q = 1.0 / np.sqrt(n_q), 1.0 / np.sqrt(d_model)
+    w_o = wl.f32_to_bf16_bits((rng.standard_normal((d_model, n_q)) * sc_o).astype(np.float32))
+    w_q = wl.f32_to_bf16_bits((rng.standard_normal((n_q, d_model)) * sc_q).astype(np.float32))
+    g = wl.f32_to_bf16_bits((1.0 + 0.1 * rng.standard_normal(d_model)).astype(np.float32))
+    a = rng.standard_normal((batch, n_q)).astype(np.float32)
+    z = wl.f32_to_bf16_bits((rng.standard_normal((batch, d_model)) * 2.0).astype(np.float32))
+    return a, z, w_o, g, w_q
+
+
+def run_gpu(a, z, w_o, g, w_q, eps):
+    batch, n_q = a.shape
+    d_model = z.shape[1]
+    need = qf.project_workspace_bytes(batch, d_model, n_q)
+    assert need > 0
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    u = torch.full((batch, d_model), float("nan"), dtype=torch.bfloat16, device="cuda")
+    q = torch.full((batch, n_q), float("nan"), dtype=torch.bfloat16, device="cuda")
+    args = (torch.from_numpy(a).cuda(), dev_bf16(z), dev_bf16(w_o), dev_bf16(g), dev_bf16(w_q), u, q, eps, ws)
+    qf.project_pair(*args)
+    torch.cuda.synchronize()
+    assert qf.project_status(ws) == 0
+    assert qf.last_launch_count() == 2
+    return host_bits(u), host_bits(q), args
+
+
+def ulp_bf16(x):
+    return 2.0 ** (np.floor(np.log2(np.maximum(np.abs(x), 2.0 ** -120))) - 7)
+
+
+def check(u, q, ref_u, ref_q, tag):
+    for name, got, ref, abs_tol, share in (("u'", u, ref_u, 1e-5, 0.01), ("q", q, ref_q, 2.5e-3, 0.05)):
+        x, r = bits_to_f64(got), bits_to_f64(ref)
+        assert np.isfinite(x).all(), (tag, name)
+        rms = np.sqrt((r ** 2).mean(axis=1, keepdims=True))
+        d = np.abs(x - r)
+        lim = ulp_bf16(np.maximum(np.abs(r), np.abs(x))) + abs_tol * rms
+        worst = np.unravel_index(np.argmax(d - lim), d.shape)
+        assert (d <= lim).all(), (tag, name, "at", worst, "got", x[worst], "ref", r[worst], "limit", lim[worst])
+        assert (d > 0).mean() < share, (tag, name, "share of elements that differ", (d > 0).mean())
+
+
+@pytest.mark.parametrize("batch,d_model,n_q", [
+    (8, 1024, 2048),      # Qwen3-0.6B shape, the paper's batch of eight
+    (1, 1024, 2048),      # served alone: the matrix-vector case
+    (17, 1024, 2048),     # a batch that is not a multiple of the tile's 16 columns
+    (8, 2560, 4096),      # Qwen3-4B shape
+    (33, 2560, 4096),     # 48 padded columns
+    (64, 2560, 4096),     # the largest batch one call takes
+    (32, 5120, 5120),     # the largest K (ten boxes per CTA)
+    (32, 512, 1024),      # the smallest shapes: one and two boxes per CTA
+])
+def test_matches_the_oracle(batch, d_model, n_q):
+    a, z, w_o, g, w_q = make_inputs(batch, d_model, n_q, seed=batch * 7 + d_model)
+    eps = 1e-6
+    u, q, _ = run_gpu(a, z, w_o, g, w_q, eps)
+    ref_u, ref_q = orc.project_pair(a, z, w_o, g, w_q, eps=eps)
+    check(u, q, ref_u, ref_q, f"batch={batch} d_model={d_model} n_q={n_q}")
+
+
+def test_structured_inputs_are_exact_and_runs_repeat_bit_for_bit():
+    batch, d_model, n_q = 8, 1024, 2048
+    a, z, w_o, g, w_q = make_inputs(batch, d_model, n_q, seed=3)
+    # one-hot attention outputs read out single columns of W_o: no rounding anywhere, so bit-exact
+    a1 = np.zeros_like(a)
+    cols = [0, 63, 64, 1023, 1024, 2047, 511, 1500]
+    for m, j in enumerate(cols):
+        a1[m, j] = 1.0
+    z0 = np.zeros_like(z)
+    u, q, args = run_gpu(a1, z0, w_o, g, w_q, 1e-6)
+    for m, j in enumerate(cols):
+        assert np.array_equal(u[m], w_o[:, j]), (m, j)
+    ref_u, ref_q = orc.project_pair(a1, z0, w_o, g, w_q, eps=1e-6)
+    check(u, q, ref_u, ref_q, "one-hot")
+    # determinism: the split-K sum runs in rank order, so repeated launches give the same bits
+    first = None
+    for _ in range(4):
+        qf.project_pair(*args)
+        torch.cuda.synchronize()
+        bits = (host_bits(args[5]).copy(), host_bits(args[6]).copy())
+        if first is None:
+            first = bits
+        assert np.array_equal(first[0], bits[0]) and np.array_equal(first[1], bits[1])
+
+
+def test_feeds_the_sweep():
+    # q of the pair has the layout the sweep consumes: project, then sweep a small cache with it
+    from paper_2608_15473_b200.runtime import DeviceWorkload
+    import qf_testlib as T
+    Hq, Hkv, D = 16, 8, 128
+    lens = [300, 4000, 17, 2048, 999, 64, 1, 1500]
+    w = wl.make_workload("proj", lens, [wl.fixed_shards(L, 1024) for L in lens], Hq, Hkv, seed=5)
+    a, z, w_o, g, w_q = make_inputs(len(lens), 1024, Hq * D, seed=11)
+    _, q_bits, _ = run_gpu(a, z, w_o, g, w_q, 1e-6)
+    w.q = q_bits.reshape(len(lens), Hq, D).copy()
+    dw = DeviceWorkload(w)
+    dw.step()
+    T.compare_all(dw, w, tag="q from the projection pair")
+
+
+def test_unsupported_shapes_and_bad_arguments_are_rejected():
+    assert qf.project_workspace_bytes(8, 1000, 2048) == 0        # not a multiple of 512
+    assert qf.project_workspace_bytes(65, 1024, 2048) == 0       # batch above 64
+    assert qf.project_workspace_bytes(64, 5120, 5120) == 0       # shared-memory budget
+    assert qf.project_workspace_bytes(64, 512, 1024) == 0        # the partial tile would not fit one weight box
+    assert qf.project_workspace_bytes(8, 1024, 6144) == 0        # K above 5,120
+    ws = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    t = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    L = qf.lib()
+    p = lambda x: qf._ptr(x)
+    assert L.qf_project_pair(p(t), p(t), p(t), p(t), p(t), p(t), p(t), 8, 1000, 2048, 1e-6, p(ws), 4096, None) == qf.QF_ERR_UNSUPPORTED
+    assert L.qf_project_pair(None, p(t), p(t), p(t), p(t), p(t), p(t), 8, 1024, 2048, 1e-6, p(ws), 4096, None) == qf.QF_ERR_NULL
+    assert L.qf_project_pair(p(t), p(t), p(t), p(t), p(t), p(t), p(t), 8, 1024, 2048, 1e-6, p(ws), 16, None) == qf.QF_ERR_WORKSPACE
+    assert L.qf_project_pair(p(t), p(t), p(t) + 64, p(t), p(t), p(t), p(t), 8, 1024, 2048, 1e-6, p(ws), 4096, None) == qf.QF_ERR_BAD_SHAPE
