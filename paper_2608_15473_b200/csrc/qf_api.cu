@@ -375,8 +375,11 @@ int qf_project_pair(const float *a, const void *z, const void *w_o, const void *
     if (rc != QF_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     CUtensorMap map_o, map_q;
-    if (qf::make_weight_map(&map_o, w_o, d_model, n_q, g_cuda_msg, sizeof g_cuda_msg)) return QF_ERR_CUDA;
-    if (qf::make_weight_map(&map_q, w_q, n_q, d_model, g_cuda_msg, sizeof g_cuda_msg)) return QF_ERR_CUDA;
+    const int np = qf::proj_padded_batch(batch);
+    const int sb_o = qf::proj_ring(n_q / (qf::kProjSplits * qf::kProjBoxK), np).sb;
+    const int sb_q = qf::proj_ring(d_model / (qf::kProjSplits * qf::kProjBoxK), np).sb;
+    if (qf::make_weight_map(&map_o, w_o, d_model, n_q, sb_o, g_cuda_msg, sizeof g_cuda_msg)) return QF_ERR_CUDA;
+    if (qf::make_weight_map(&map_q, w_q, n_q, d_model, sb_q, g_cuda_msg, sizeof g_cuda_msg)) return QF_ERR_CUDA;
     unsigned *status = (unsigned *)workspace;
     float *ssq_part = (float *)((char *)workspace + 256);
 

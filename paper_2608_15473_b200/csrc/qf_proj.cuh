@@ -10,9 +10,14 @@
 //     tcgen05.mma (128 output features per CTA), the batch is the N side (16..64 columns), the
 //     accumulator lives in tensor memory.
 //   * K is split eight ways over a thread-block cluster, so a 2,560 x 4,096 weight keeps 160 CTAs busy;
-//     a CTA's whole weight slice (128 x K/8 bf16) is requested by TMA at the very start of the kernel,
-//     before the programmatic dependency on the previous kernel is waited for (weights are never
-//     produced on the path), and is consumed box by box as it lands.
+//     a CTA's weight slice (128 x K/8 bf16) streams through a small ring of TMA requests, each of several
+//     adjacent 128-row x 128-byte boxes (so that a request reads 256 bytes to 1 KB contiguous per weight row:
+//     with one 128-byte box per request every row segment opened its own DRAM page and the stream ran at
+//     a third of the HBM rate); the ring's first fill is requested at the very start of the kernel, before the programmatic dependency on the
+//     previous kernel is waited for (weights are never produced on the path); a slot is refilled as soon
+//     as the products that read it have completed (tcgen05.commit on the slot's barrier).  The ring, not
+//     the whole slice, is resident so that two CTAs fit an SM and every cluster of a product is resident
+//     at once: with the whole slice resident the kernel ran in two waves and took twice as long.
 //   * the eight partial tiles are summed over distributed shared memory in rank order (bit-deterministic),
 //     each rank finishing 16 of the tile's 128 output features.
 //
@@ -41,6 +46,7 @@ constexpr int kProjTileOut   = 128;   // output features per CTA = rows of the t
 constexpr int kProjSplits    = 8;     // K splits = CTAs of a cluster
 constexpr int kProjBoxK      = 64;    // bf16 per TMA box row: 128 bytes, one swizzle span
 constexpr int kProjMaxBoxes  = 10;    // K / 8 / 64 <= 10, i.e. K <= 5,120
+constexpr int kProjMaxRing   = 4;     // weight boxes in flight per CTA
 constexpr int kProjMaxBatch  = 64;
 constexpr int kProjRowsPerRank = kProjTileOut / kProjSplits;   // 16
 
@@ -54,6 +60,7 @@ struct ProjArgs {
     unsigned *status;          // bit 1 (QF_STATUS_TIMEOUT) is ORed in when a wait runs out
     int batch, n_out, k_total;
     int ssq_tiles;             // stage 1: number of stage 0 tiles
+    int ring_sb, ring_slots;   // boxes per TMA request, requests in flight per CTA (proj_ring)
     float inv_d_model, eps;    // stage 1
 };
 
@@ -113,13 +120,15 @@ __device__ __forceinline__ float ld_peer_f32(uint32_t local_smem_addr, uint32_t 
     asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
     return v;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar,
-                                            unsigned long long policy)
+// One request: `sb` adjacent boxes (the map's box is [sb column blocks][128 rows][64 bf16]) starting at weight
+// row `row` and column block `kblock`; they land as sb consecutive swizzled [128][128 B] tiles.
+__device__ __forceinline__ void tma_load_boxes(uint32_t dst, const CUtensorMap *map, int row, int kblock, uint32_t bar,
+                                               unsigned long long policy)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
-        " [%0], [%1, {%2, %3}], [%4], %5;"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(kblock), "r"(bar), "l"(policy) : "memory");
 }
 
 // Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes, 128B-swizzled, eight-row
@@ -136,22 +145,47 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-// Dynamic shared memory: this header (1 KB), then n_boxes weight boxes [128 rows][128 B], then n_boxes
+// Dynamic shared memory: this header (2 KB), then a ring of weight boxes [128 rows][128 B], then n_boxes
 // activation boxes [NP rows][128 B]; every box is 1,024-byte aligned.  The partial tile [NP][128] fp32
-// reuses the weight boxes once the products are done (the host checks that it fits).
+// reuses the ring once the products are done (the host checks that it fits).
 struct ProjSmemHeader {
-    alignas(8) unsigned long long w_full[kProjMaxBoxes];
+    alignas(8) unsigned long long w_full[kProjMaxRing];    // a slot's box has landed
+    alignas(8) unsigned long long w_empty[kProjMaxRing];   // the products reading a slot have completed
     alignas(8) unsigned long long mma_done;
     uint32_t tmem_base;
     int abort_flag;
     float ssq[kProjMaxBatch];      // stage 0: this rank's sums of squares; stage 1: 1/rms per request
     float half_sum[kProjMaxBatch]; // stage 1 prologue
+    alignas(16) uint16_t gain[kProjMaxBoxes * kProjBoxK];   // stage 1: this K slice of g
 };
-static_assert(sizeof(ProjSmemHeader) <= 1024, "header must fit its kilobyte");
+constexpr int kProjHeaderBytes = 2048;
+static_assert(sizeof(ProjSmemHeader) <= kProjHeaderBytes, "header must fit its two kilobytes");
 constexpr int kProjWBoxBytes = kProjTileOut * 128;
-inline size_t proj_smem_bytes(int n_boxes, int np)
+inline size_t proj_smem_bytes(int ring, int n_boxes, int np)
 {
-    return 1024 /* alignment slack */ + 1024 + (size_t)n_boxes * (kProjWBoxBytes + np * 128);
+    return 1024 /* alignment slack */ + kProjHeaderBytes + (size_t)ring * kProjWBoxBytes + (size_t)n_boxes * np * 128;
+}
+// The ring: `slots` requests in flight, each of `sb` adjacent boxes (sb divides the slice's box count).
+// Preferred: the largest request that still leaves room for two CTAs per SM (then every cluster of a product
+// is resident at once), with at least two slots unless one request covers the whole slice; the ring must also
+// hold the partial tile.  Falls back to one CTA per SM when nothing smaller fits.
+struct ProjRing { int sb, slots; };
+inline ProjRing proj_ring(int n_boxes, int np)
+{
+    const int need = (np * kProjTileOut * 4 + kProjWBoxBytes - 1) / kProjWBoxBytes;   // boxes the partial tile covers
+    for (int pass = 0; pass < 2; ++pass) {
+        const size_t budget = (pass == 0 ? 113 : 227) * 1024;
+        for (int sb = n_boxes; sb >= 1; --sb) {
+            if (n_boxes % sb) continue;
+            const int n_req = n_boxes / sb;
+            for (int slots = (n_req < kProjMaxRing ? n_req : kProjMaxRing); slots >= 1; --slots) {
+                if (slots == 1 && n_req > 1) break;
+                if (sb * slots < need) break;
+                if (proj_smem_bytes(sb * slots, n_boxes, np) <= budget) return ProjRing{sb, slots};
+            }
+        }
+    }
+    return ProjRing{0, 0};
 }
 
 template <int STAGE, int NP>
@@ -165,22 +199,31 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
     const int rank = (int)cluster_rank();                 // which eighth of K
     const int tile = (int)blockIdx.x / kProjSplits;       // which 128 output features
     const int k_slice = A.k_total / kProjSplits, n_boxes = k_slice / kProjBoxK;
-    uint8_t *w_boxes = smem_al + 1024;                    // [n_boxes][128][128 B]
-    uint8_t *x_boxes = w_boxes + (size_t)n_boxes * kProjWBoxBytes;   // [n_boxes][NP][128 B]
+    const int sb = A.ring_sb, slots = A.ring_slots, n_req = n_boxes / sb;   // boxes per request, requests in flight, requests
+    uint8_t *w_boxes = smem_al + kProjHeaderBytes;        // [slots][sb][128][128 B]
+    uint8_t *x_boxes = w_boxes + (size_t)slots * sb * kProjWBoxBytes;   // [n_boxes][NP][128 B]
     const int k0 = rank * k_slice;
     volatile int *abort_flag = &sm.abort_flag;
 
-    if (tid == 0) {
-        for (int i = 0; i < n_boxes; ++i) mbar_init(smem_u32(&sm.w_full[i]), 1);
+    // thread 32 owns the weight stream and the products
+    const unsigned long long policy = l2_evict_first_policy();
+    auto issue_req = [&](int r) {   // request r: boxes [r sb, r sb + sb) of this CTA's slice
+        const int slot = r % slots;
+        mbar_arrive_expect_tx(smem_u32(&sm.w_full[slot]), (uint32_t)sb * kProjWBoxBytes);
+        tma_load_boxes(smem_u32(w_boxes + (size_t)slot * sb * kProjWBoxBytes), &w_map, tile * kProjTileOut,
+                       k0 / kProjBoxK + r * sb, smem_u32(&sm.w_full[slot]), policy);
+    };
+    int issued = 0;
+    if (tid == 32) {
+        for (int i = 0; i < slots; ++i) {
+            mbar_init(smem_u32(&sm.w_full[i]), 1);
+            mbar_init(smem_u32(&sm.w_empty[i]), 1);
+        }
         mbar_init(smem_u32(&sm.mma_done), 1);
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        // the whole weight slice, now: it does not depend on anything the stream computed before
-        const unsigned long long policy = l2_evict_first_policy();
-        for (int i = 0; i < n_boxes; ++i) {
-            mbar_arrive_expect_tx(smem_u32(&sm.w_full[i]), kProjTileOut * 128);
-            tma_load_2d(smem_u32(w_boxes + (size_t)i * kProjWBoxBytes), &w_map, k0 + i * kProjBoxK, tile * kProjTileOut, smem_u32(&sm.w_full[i]), policy);
-        }
+        // the first fill of the ring, now: the weight does not depend on anything the stream computed before
+        for (; issued < slots; ++issued) issue_req(issued);
     }
     if (warp == 0) tmem_alloc(smem_u32(&sm.tmem_base), 64);
 
@@ -188,44 +231,114 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
     grid_launch_dependents();
     if (STAGE == 0 && blockIdx.x == 0 && tid == 0) *A.status = 0u;
 
-    // ---- activations of this K slice, as the B operand: [NP rows][k_slice] bf16, 128B-swizzled boxes
-    if (STAGE == 1) {
-        // 1/rms per request from stage 0's per-tile sums of squares, summed in tile order (two interleaved halves)
-        const int n = tid & (kProjMaxBatch - 1), half = tid / kProjMaxBatch;
-        float s = 0.f;
-        if (n < A.batch)
-            for (int p = half; p < A.ssq_tiles; p += 2) s += ld_sync_f32(A.ssq_part + (size_t)p * kProjMaxBatch + n);
-        if (half == 1) sm.half_sum[n] = s;
-        __syncthreads();
-        if (half == 0) sm.ssq[n] = 1.0f / sqrtf((s + sm.half_sum[n]) * A.inv_d_model + A.eps);
-        __syncthreads();
+    // ---- activations of this K slice, as the B operand: [NP rows][k_slice] bf16, 128B-swizzled boxes.
+    // Global loads are issued eight items at a time per thread before any of them is used (the prologue is
+    // a few dependent round trips to L2 long; done one by one it was longer than streaming the weight).
+    constexpr int kU = 8;
+    const int chunks_per_row = k_slice / 8;               // 16-byte chunks of 8 bf16
+    const int n_items = A.batch * chunks_per_row;         // rows at or beyond the batch are zero-filled below
+    auto item_addr = [&](int idx, int &m, int &k) { m = idx / chunks_per_row; k = (idx - m * chunks_per_row) * 8; };
+    auto x_slot = [&](int m, int k) -> uint4 * {
+        const int box = k / kProjBoxK, c = (k % kProjBoxK) / 8;
+        return reinterpret_cast<uint4 *>(x_boxes + (size_t)box * (NP * 128) + m * 128 + ((c ^ (m & 7)) * 16));
+    };
+    // what the epilogue adds to the product (stage 0), fetched now so that it has long arrived by then
+    const int ep_j = tid & (kProjRowsPerRank - 1), ep_n0 = tid / kProjRowsPerRank;
+    const int ep_o = tile * kProjTileOut + rank * kProjRowsPerRank + ep_j;
+    uint16_t zreg[NP / 8];
+#pragma unroll
+    for (int i = 0; i < NP / 8; ++i) {
+        const int n = ep_n0 + 8 * i;
+        zreg[i] = (STAGE == 0 && n < A.batch) ? A.z[(size_t)n * A.n_out + ep_o] : (uint16_t)0;
     }
-    {
-        const int chunks_per_row = k_slice / 8;           // 16-byte chunks of 8 bf16
-        for (int idx = tid; idx < NP * chunks_per_row; idx += kProjThreads) {
-            const int m = idx / chunks_per_row, ck = idx - m * chunks_per_row;
-            const int k = ck * 8, box = k / kProjBoxK, c = (k % kProjBoxK) / 8;
-            uint4 pk = make_uint4(0u, 0u, 0u, 0u);
-            if (m < A.batch) {
-                if (STAGE == 0) {
-                    const float4 lo = *reinterpret_cast<const float4 *>(A.a + (size_t)m * A.k_total + k0 + k);
-                    const float4 hi = *reinterpret_cast<const float4 *>(A.a + (size_t)m * A.k_total + k0 + k + 4);
-                    pk = make_uint4(pack_bf16(lo.x, lo.y), pack_bf16(lo.z, lo.w), pack_bf16(hi.x, hi.y), pack_bf16(hi.z, hi.w));
-                } else {
-                    const uint4 uw = *reinterpret_cast<const uint4 *>(A.u_in + (size_t)m * A.k_total + k0 + k);
-                    const uint4 gw = *reinterpret_cast<const uint4 *>(A.g + k0 + k);
+    if (STAGE == 0) {
+        for (int base = tid; base < n_items; base += kProjThreads * kU) {
+            float4 lo[kU], hi[kU];
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                const int idx = base + u * kProjThreads;
+                if (idx < n_items) {
+                    int m, k;
+                    item_addr(idx, m, k);
+                    const float *src = A.a + (size_t)m * A.k_total + k0 + k;
+                    lo[u] = *reinterpret_cast<const float4 *>(src);
+                    hi[u] = *reinterpret_cast<const float4 *>(src + 4);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                const int idx = base + u * kProjThreads;
+                if (idx < n_items) {
+                    int m, k;
+                    item_addr(idx, m, k);
+                    *x_slot(m, k) = make_uint4(pack_bf16(lo[u].x, lo[u].y), pack_bf16(lo[u].z, lo[u].w),
+                                               pack_bf16(hi[u].x, hi[u].y), pack_bf16(hi[u].z, hi[u].w));
+                }
+            }
+        }
+    } else {
+        // the gain slice and the first batch of the stream go out before the sums of squares are waited for
+        for (int i = tid; i < k_slice / 8; i += kProjThreads)
+            reinterpret_cast<uint4 *>(sm.gain)[i] = *reinterpret_cast<const uint4 *>(A.g + k0 + i * 8);
+        uint4 uw[kU];
+        auto load_batch = [&](int base) {
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                const int idx = base + u * kProjThreads;
+                if (idx < n_items) {
+                    int m, k;
+                    item_addr(idx, m, k);
+                    uw[u] = *reinterpret_cast<const uint4 *>(A.u_in + (size_t)m * A.k_total + k0 + k);
+                }
+            }
+        };
+        load_batch(tid);
+        {
+            // 1/rms per request from stage 0's per-tile sums of squares, summed in tile order (two interleaved halves)
+            const int n = tid & (kProjMaxBatch - 1), half = tid / kProjMaxBatch;
+            float s = 0.f;
+            if (n < A.batch) {
+                for (int p0 = half; p0 < A.ssq_tiles; p0 += 2 * kU) {
+                    float v[kU];
+#pragma unroll
+                    for (int u = 0; u < kU; ++u) {
+                        const int p = p0 + 2 * u;
+                        v[u] = (p < A.ssq_tiles) ? ld_sync_f32(A.ssq_part + (size_t)p * kProjMaxBatch + n) : 0.f;
+                    }
+#pragma unroll
+                    for (int u = 0; u < kU; ++u) s += v[u];
+                }
+            }
+            if (half == 1) sm.half_sum[n] = s;
+            __syncthreads();
+            if (half == 0) sm.ssq[n] = 1.0f / sqrtf((s + sm.half_sum[n]) * A.inv_d_model + A.eps);
+            __syncthreads();
+        }
+        for (int base = tid; base < n_items; base += kProjThreads * kU) {
+            if (base != tid) load_batch(base);
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                const int idx = base + u * kProjThreads;
+                if (idx < n_items) {
+                    int m, k;
+                    item_addr(idx, m, k);
+                    const uint4 gw = *reinterpret_cast<const uint4 *>(sm.gain + k);
                     const float r = sm.ssq[m];
-                    const uint32_t uu[4] = {uw.x, uw.y, uw.z, uw.w}, gg[4] = {gw.x, gw.y, gw.z, gw.w};
+                    const uint32_t uu[4] = {uw[u].x, uw[u].y, uw[u].z, uw[u].w}, gg[4] = {gw.x, gw.y, gw.z, gw.w};
                     uint32_t o[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e)   // g*u is exact in fp32 (two bf16 factors); one rounding by r, one to bf16
                         o[e] = pack_bf16(bf16lo_to_f32(gg[e]) * bf16lo_to_f32(uu[e]) * r,
                                          bf16hi_to_f32(gg[e]) * bf16hi_to_f32(uu[e]) * r);
-                    pk = make_uint4(o[0], o[1], o[2], o[3]);
+                    *x_slot(m, k) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
             }
-            *reinterpret_cast<uint4 *>(x_boxes + (size_t)box * (NP * 128) + m * 128 + ((c ^ (m & 7)) * 16)) = pk;
         }
+    }
+    for (int idx = n_items + tid; idx < NP * chunks_per_row; idx += kProjThreads) {   // padding rows
+        int m, k;
+        item_addr(idx, m, k);
+        *x_slot(m, k) = make_uint4(0u, 0u, 0u, 0u);
     }
     // the tensor core reads shared memory through the async proxy: make the stores above visible to it
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -234,18 +347,31 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&sm.tmem_base);
 
-    // ---- products: one thread issues them box by box as the weight lands
+    // ---- products: thread 32 issues them box by box as the weight lands, and refills the slots behind them
     if (tid == 32) {
         constexpr uint32_t idesc = umma_idesc_bf16(NP);
         bool ok = true;
-        for (int i = 0; i < n_boxes && ok; ++i) {
-            if (!mbar_wait(smem_u32(&sm.w_full[i]), 0, abort_flag)) { ok = false; break; }
+        int consumed = 0;
+        for (int r = 0; r < n_req; ++r) {
+            const int slot = r % slots;
+            if (!mbar_wait(smem_u32(&sm.w_full[slot]), (uint32_t)((r / slots) & 1), abort_flag)) { ok = false; break; }
+            consumed = r + 1;
             tc_fence_after();
-            const uint64_t ad = umma_desc_k_sw128(smem_u32(w_boxes + (size_t)i * kProjWBoxBytes));
-            const uint64_t bd = umma_desc_k_sw128(smem_u32(x_boxes + (size_t)i * (NP * 128)));
+            for (int j = 0; j < sb; ++j) {
+                const int i = r * sb + j;     // box of the slice
+                const uint64_t ad = umma_desc_k_sw128(smem_u32(w_boxes + (size_t)(slot * sb + j) * kProjWBoxBytes));
+                const uint64_t bd = umma_desc_k_sw128(smem_u32(x_boxes + (size_t)i * (NP * 128)));
 #pragma unroll
-            for (int kk = 0; kk < kProjBoxK / 16; ++kk)   // 16 bf16 = 32 bytes = 2 descriptor units along K
-                umma_bf16(tmem, ad + 2 * kk, bd + 2 * kk, idesc, (i | kk) ? 1u : 0u);
+                for (int kk = 0; kk < kProjBoxK / 16; ++kk)   // 16 bf16 = 32 bytes = 2 descriptor units along K
+                    umma_bf16(tmem, ad + 2 * kk, bd + 2 * kk, idesc, (i | kk) ? 1u : 0u);
+            }
+            umma_commit(smem_u32(&sm.w_empty[slot]));     // arrives when the products above have completed
+            // refill the slot of the request before this one: its products have had this iteration to complete
+            if (r >= 1 && issued < n_req) {
+                const int ps = (r - 1) % slots;
+                if (!mbar_wait(smem_u32(&sm.w_empty[ps]), (uint32_t)(((r - 1) / slots) & 1), abort_flag)) { ok = false; break; }
+                issue_req(issued++);
+            }
         }
         if (ok) {
             umma_commit(smem_u32(&sm.mma_done));
@@ -253,9 +379,9 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
             sm.abort_flag = 1;
             atomicOr(A.status, (unsigned)kStatusTimeout);
             // copies still in flight must land before this CTA's shared memory goes away
-            for (int i = 0; i < n_boxes; ++i)
+            for (int r = consumed; r < issued; ++r)
                 for (unsigned it = 0; it < (1u << 20); ++it)
-                    if (mbar_try_wait(smem_u32(&sm.w_full[i]), 0)) break;
+                    if (mbar_try_wait(smem_u32(&sm.w_full[r % slots]), (uint32_t)((r / slots) & 1))) break;
             mbar_arrive(smem_u32(&sm.mma_done));
         }
     }
@@ -282,34 +408,38 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
 
     // ---- sum the eight partials in rank order; this rank finishes output features [16 rank, 16 rank + 16)
     {
-        const int j = tid & (kProjRowsPerRank - 1), n0 = tid / kProjRowsPerRank;   // feature within the rank's 16, request lane
-        const int o = tile * kProjTileOut + rank * kProjRowsPerRank + j;
         const uint32_t part_addr = smem_u32(part);
+        float pv[NP / 8][kProjSplits];
 #pragma unroll
-        for (int i = 0; i < NP / 8; ++i) {
-            const int n = n0 + 8 * i;
-            float y = 0.f;
+        for (int i = 0; i < NP / 8; ++i)        // every remote read is issued before any is summed
 #pragma unroll
             for (int c = 0; c < kProjSplits; ++c)
-                y += ld_peer_f32(part_addr + (uint32_t)((n * kProjTileOut + rank * kProjRowsPerRank + j) * 4), (uint32_t)c);
+                pv[i][c] = ld_peer_f32(part_addr + (uint32_t)(((ep_n0 + 8 * i) * kProjTileOut + rank * kProjRowsPerRank + ep_j) * 4),
+                                       (uint32_t)c);
+#pragma unroll
+        for (int i = 0; i < NP / 8; ++i) {
+            const int n = ep_n0 + 8 * i;
+            float y = 0.f;
+#pragma unroll
+            for (int c = 0; c < kProjSplits; ++c) y += pv[i][c];
             float sq = 0.f;
             if (n < A.batch) {
                 if (STAGE == 0) {
-                    const float zf = __uint_as_float((uint32_t)A.z[(size_t)n * A.n_out + o] << 16);
+                    const float zf = __uint_as_float((uint32_t)zreg[i] << 16);
                     const __nv_bfloat16 ub = __float2bfloat16_rn(zf + y);
-                    A.out[(size_t)n * A.n_out + o] = *reinterpret_cast<const uint16_t *>(&ub);
+                    A.out[(size_t)n * A.n_out + ep_o] = *reinterpret_cast<const uint16_t *>(&ub);
                     const float uf = __bfloat162float(ub);
                     sq = uf * uf;
                 } else {
                     const __nv_bfloat16 qb = __float2bfloat16_rn(y);
-                    A.out[(size_t)n * A.n_out + o] = *reinterpret_cast<const uint16_t *>(&qb);
+                    A.out[(size_t)n * A.n_out + ep_o] = *reinterpret_cast<const uint16_t *>(&qb);
                 }
             }
             if (STAGE == 0) {
                 // sum of squares over the rank's 16 features: the 16 lanes of a half warp, fixed tree
 #pragma unroll
                 for (int off = 8; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
-                if (j == 0) sm.ssq[n] = sq;
+                if (ep_j == 0) sm.ssq[n] = sq;
             }
         }
     }
@@ -328,20 +458,21 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
 }
 
 // ------------------------------------------------------------------ host side
-// A [rows][cols] row-major bf16 weight as 128B-swizzled boxes of 128 rows x 64 columns.
-inline int make_weight_map(CUtensorMap *out, const void *w, int rows, int cols, char *msg, size_t msg_len)
+// A [rows][cols] row-major bf16 weight seen as [cols / 64 column blocks][rows][64]: a box is sb adjacent column
+// blocks of 128 rows, each landing as a 128B-swizzled [128][128 B] tile.
+inline int make_weight_map(CUtensorMap *out, const void *w, int rows, int cols, int sb, char *msg, size_t msg_len)
 {
     typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
     static EncodeFn encode = nullptr;
     static std::mutex mu;
-    struct Entry { const void *w; int rows, cols; CUtensorMap map; };
+    struct Entry { const void *w; int rows, cols, sb; CUtensorMap map; };
     static Entry cache[32];
     static int n_cached = 0, next = 0;
     std::lock_guard<std::mutex> lock(mu);
     for (int i = 0; i < n_cached; ++i)
-        if (cache[i].w == w && cache[i].rows == rows && cache[i].cols == cols) {
+        if (cache[i].w == w && cache[i].rows == rows && cache[i].cols == cols && cache[i].sb == sb) {
             *out = cache[i].map;
             return 0;
         }
@@ -355,12 +486,12 @@ inline int make_weight_map(CUtensorMap *out, const void *w, int rows, int cols, 
         }
         encode = (EncodeFn)fn;
     }
-    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kProjBoxK, (cuuint32_t)kProjTileOut};
-    const cuuint32_t estr[2] = {1, 1};
+    const cuuint64_t dims[3] = {(cuuint64_t)kProjBoxK, (cuuint64_t)rows, (cuuint64_t)(cols / kProjBoxK)};
+    const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)kProjBoxK * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)kProjBoxK, (cuuint32_t)kProjTileOut, (cuuint32_t)sb};
+    const cuuint32_t estr[3] = {1, 1, 1};
     CUtensorMap map;
-    CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(w), dims, strides, box, estr,
+    CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(w), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -368,7 +499,7 @@ inline int make_weight_map(CUtensorMap *out, const void *w, int rows, int cols, 
         return -1;
     }
     Entry &slot = cache[next];
-    slot.w = w; slot.rows = rows; slot.cols = cols; slot.map = map;
+    slot.w = w; slot.rows = rows; slot.cols = cols; slot.sb = sb; slot.map = map;
     next = (next + 1) % 32;
     if (n_cached < 32) ++n_cached;
     *out = map;
@@ -384,17 +515,28 @@ inline bool proj_shape_ok(int batch, int n_out, int k_total)
     if (batch < 1 || batch > kProjMaxBatch || n_out < kProjTileOut || n_out % kProjTileOut) return false;
     if (k_total % (kProjSplits * kProjBoxK) || k_total / (kProjSplits * kProjBoxK) > kProjMaxBoxes) return false;
     const int np = proj_padded_batch(batch), n_boxes = k_total / (kProjSplits * kProjBoxK);
-    if ((size_t)np * kProjTileOut * 4 > (size_t)n_boxes * kProjWBoxBytes) return false;   // partial tile reuses the weight boxes
-    return proj_smem_bytes(n_boxes, np) <= 227 * 1024;
+    return proj_ring(n_boxes, np).slots > 0;
 }
 
 template <int STAGE, int NP>
 cudaError_t launch_proj_np(const CUtensorMap &map, const ProjArgs &args, cudaStream_t st)
 {
     const int n_boxes = args.k_total / (kProjSplits * kProjBoxK);
-    const size_t smem = proj_smem_bytes(n_boxes, NP);
-    cudaError_t e = cudaFuncSetAttribute(proj_kernel<STAGE, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
+    const ProjRing ring = proj_ring(n_boxes, NP);
+    ProjArgs a2 = args;
+    a2.ring_sb = ring.sb;
+    a2.ring_slots = ring.slots;
+    const size_t smem = proj_smem_bytes(ring.sb * ring.slots, n_boxes, NP);
+    // the attribute is raised once per device to the largest footprint this instantiation can have
+    static bool attr_set[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_set[dev & 63]) {
+        cudaError_t ea = cudaFuncSetAttribute(proj_kernel<STAGE, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              227 * 1024);
+        if (ea != cudaSuccess) return ea;
+        attr_set[dev & 63] = true;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(args.n_out / kProjTileOut * kProjSplits));
     cfg.blockDim = dim3(kProjThreads);
@@ -409,7 +551,7 @@ cudaError_t launch_proj_np(const CUtensorMap &map, const ProjArgs &args, cudaStr
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, proj_kernel<STAGE, NP>, map, args);
+    return cudaLaunchKernelEx(&cfg, proj_kernel<STAGE, NP>, map, a2);
 }
 template <int STAGE>
 cudaError_t launch_proj(const CUtensorMap &map, const ProjArgs &args, cudaStream_t st)
