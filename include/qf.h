@@ -225,7 +225,11 @@ int qf_append_kv(void *k_cache, void *v_cache, const int32_t *block_table, const
  * Supported: 1 <= batch <= 64; d_model and n_q multiples of 512, at most
  * 5,120 (for batch > 32: at least 1,024); else
  * QF_ERR_UNSUPPORTED (qf_project_workspace_bytes returns 0).  Larger batches
- * are run in slices of 64 by the caller.  Enqueues two kernels on cuda_stream.
+ * are run in slices of 64 by the caller.  Enqueues two kernels on cuda_stream
+ * (capturable in a CUDA graph; the first call for a shape sets kernel
+ * attributes and builds the weights' TMA descriptors, so make one call
+ * before capturing).  Meant for the paper's regime of a few co-resident
+ * requests: from a batch of about 32 on a library GEMM is as fast or faster.
  * qf_project_status copies the pair's status word (QF_STATUS_TIMEOUT if a
  * bounded wait inside a kernel ran out; 0 = clean) and synchronises the stream.
  */

@@ -155,3 +155,28 @@ def test_unsupported_shapes_and_bad_arguments_are_rejected():
     assert L.qf_project_pair(None, p(t), p(t), p(t), p(t), p(t), p(t), 8, 1024, 2048, 1e-6, p(ws), 4096, None) == qf.QF_ERR_NULL
     assert L.qf_project_pair(p(t), p(t), p(t), p(t), p(t), p(t), p(t), 8, 1024, 2048, 1e-6, p(ws), 16, None) == qf.QF_ERR_WORKSPACE
     assert L.qf_project_pair(p(t), p(t), p(t) + 64, p(t), p(t), p(t), p(t), 8, 1024, 2048, 1e-6, p(ws), 4096, None) == qf.QF_ERR_BAD_SHAPE
+
+
+def test_graph_replay_with_new_inputs():
+    # the pair captured in a CUDA graph and replayed with new attention outputs: every replay is a fresh call
+    batch, d_model, n_q = 8, 1024, 2048
+    a, z, w_o, g, w_q = make_inputs(batch, d_model, n_q, seed=21)
+    _, _, args = run_gpu(a, z, w_o, g, w_q, 1e-6)           # first call outside capture
+    a_dev, u_dev, q_dev = args[0], args[5], args[6]
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            qf.project_pair(*args, stream=s)
+    rng = np.random.default_rng(22)
+    for it in range(3):
+        a2 = rng.standard_normal(a.shape).astype(np.float32)
+        a_dev.copy_(torch.from_numpy(a2).cuda())
+        u_dev.fill_(float("nan"))
+        q_dev.fill_(float("nan"))
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        ref_u, ref_q = orc.project_pair(a2, z, w_o, g, w_q, eps=1e-6)
+        check(host_bits(u_dev), host_bits(q_dev), ref_u, ref_q, f"replay {it}")
+        assert qf.project_status(args[8]) == 0
