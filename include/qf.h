@@ -112,7 +112,7 @@ enum {
 
 typedef struct qf_params {
     int32_t batch;             /* B                                              */
-    int32_t num_q_heads;       /* Hq                                             */
+    int32_t num_q_heads;       /* Hq: a multiple of Hkv, group G = Hq/Hkv in 1..8 */
     int32_t num_kv_heads;      /* Hkv                                            */
     int32_t head_dim;          /* D, must be 128                                 */
     int32_t page_size;         /* must be 16                                     */

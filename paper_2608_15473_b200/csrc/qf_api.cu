@@ -35,7 +35,7 @@ int validate(const qf_params *p)
     if (p->num_q_heads % p->num_kv_heads) return QF_ERR_BAD_SHAPE;
     if (p->head_dim != qf::kHeadDim || p->page_size != qf::kPageSize) return QF_ERR_UNSUPPORTED;
     const int G = p->num_q_heads / p->num_kv_heads;
-    if (G != 1 && G != 2 && G != 4 && G != 8) return QF_ERR_UNSUPPORTED;
+    if (G < 1 || G > 8) return QF_ERR_UNSUPPORTED;
     // grid dimensions and 32-bit unit counts of the sweep plan
     if (p->batch > 65535 || p->num_kv_heads > 65535) return QF_ERR_UNSUPPORTED;
     if ((long long)p->batch * p->max_shards * p->num_kv_heads > (1ll << 22)) return QF_ERR_UNSUPPORTED;
@@ -112,7 +112,7 @@ const char *qf_strerror(int status)
     case QF_OK: return "ok";
     case QF_ERR_NULL: return "a required pointer is NULL";
     case QF_ERR_BAD_SHAPE: return "bad shape: sizes must be positive and num_q_heads a multiple of num_kv_heads";
-    case QF_ERR_UNSUPPORTED: return "unsupported: head_dim must be 128, page_size 16, group size 1, 2, 4 or 8";
+    case QF_ERR_UNSUPPORTED: return "unsupported: head_dim must be 128, page_size 16, group size 1 to 8";
     case QF_ERR_WORKSPACE: return "workspace is NULL, not 256-byte aligned, or too small";
     case QF_ERR_CUDA: return g_cuda_msg[0] ? g_cuda_msg : "CUDA error";
     case QF_ERR_DEVICE: return "device is not compute capability 10.x (this library is built for sm_100a only)";
@@ -163,7 +163,11 @@ int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache, c
         switch (P.group) {
         case 1: return launch_simple<1>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, header, epoch, st);
         case 2: return launch_simple<2>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, header, epoch, st);
+        case 3: return launch_simple<3>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, header, epoch, st);
         case 4: return launch_simple<4>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, header, epoch, st);
+        case 5: return launch_simple<5>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, header, epoch, st);
+        case 6: return launch_simple<6>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, header, epoch, st);
+        case 7: return launch_simple<7>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, header, epoch, st);
         default: return launch_simple<8>(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P, header, epoch, st);
         }
     }

@@ -351,121 +351,121 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             return block_table ? block_table[rb + lp] : (int)(rb + lp);
         };
         for (;;) {   // pieces: the static slice, then chunks drawn from the counter
-        int pos, pos1;
-        piece_range(pg, n_ctas, piece, pos, pos1);
-        // the next chunk is drawn two stages before this piece's last issue: late enough that a slow SM
-        // does not sit on a reserved chunk, early enough that the counter's latency is hidden
-        const int draw_at = max(pos, pos1 - 2);
-        unsigned long long drawn = 0;
-        if (pg.n_chunks > 0 && pos >= pos1 && lane == 0) drawn = atomicAdd(header + kHdrChunk, 1ull);
-        // Every piece leaves one record for the finish kernel: the unit it must merge, if any (see below).
-        const int piece_pos0 = pos;
-        if (pos >= pos1 && lane == 0) piece_info[piece] = make_int4(-1, 0, 0, (int)(unsigned)epoch);
-        if (pos < pos1) {  // largest e with prefix[e] <= pos (pieces are drawn in increasing order)
-            int lo = e, hi = n_entries;
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (prefix[mid] <= pos) lo = mid; else hi = mid;
-            }
-            e = lo;
-        }
-        while (ok && pos < pos1) {
-            while (prefix[e + 1] <= pos) ++e;  // skip empty entries
-            const int base = prefix[e];
-            const int nunits = (prefix[e + 1] - base) / Hkv;
-            const int r = pos - base;
-            const int c = r / nunits, j = r - c * nunits;
-            const int seg_len = min(nunits - j, pos1 - pos);
-            const int b = e / S;
-            if (e != cur_e) {
-                if (e == nxt_e) clamp_range(nxt_r0, nxt_r1, nxt_len, beg, end);
-                else clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[b], beg, end);
-                cur_e = e;
-                if (e == nxt_tbl_e) { head_tbl = nxt_tbl; head_tbl_e = e; }
-                // start fetching the next non-empty shard's range; it is consumed a segment later
-                int e2 = e + 1;
-                while (e2 < n_entries && prefix[e2 + 1] == prefix[e2]) ++e2;
-                nxt_e = -1;
-                if (e2 < n_entries && prefix[e2] < pos1) {
-                    nxt_e = e2;
-                    nxt_r0 = shard_ranges[2 * e2];
-                    nxt_r1 = shard_ranges[2 * e2 + 1];
-                    nxt_len = seq_lens[e2 / S];
+            int pos, pos1;
+            piece_range(pg, n_ctas, piece, pos, pos1);
+            // the next chunk is drawn two stages before this piece's last issue: late enough that a slow SM
+            // does not sit on a reserved chunk, early enough that the counter's latency is hidden
+            const int draw_at = max(pos, pos1 - 2);
+            unsigned long long drawn = 0;
+            if (pg.n_chunks > 0 && pos >= pos1 && lane == 0) drawn = atomicAdd(header + kHdrChunk, 1ull);
+            // Every piece leaves one record for the finish kernel: the unit it must merge, if any (see below).
+            const int piece_pos0 = pos;
+            if (pos >= pos1 && lane == 0) piece_info[piece] = make_int4(-1, 0, 0, (int)(unsigned)epoch);
+            if (pos < pos1) {  // largest e with prefix[e] <= pos (pieces are drawn in increasing order)
+                int lo = e, hi = n_entries;
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (prefix[mid] <= pos) lo = mid; else hi = mid;
                 }
+                e = lo;
             }
-            const int first_page = beg >> 4, last_page = (end - 1) >> 4;
-            // the pieces that touch this unit: one segment each, slot = unit + piece (both increase along
-            // the unit space, so no two segments share a slot)
-            const int p0 = base + c * nunits;
-            const int first_piece = piece_of(pg, n_ctas, p0), last_piece = piece_of(pg, n_ctas, p0 + nunits - 1);
-            const int nseg = last_piece - first_piece + 1;
-            const int first_slot = e * Hkv + c + first_piece;
-            if (pos == piece_pos0 && lane == 0)   // does this piece start inside a unit?  (the finish kernel's input)
-                piece_info[piece] = make_int4(j > 0 ? e * Hkv + c : -1, first_slot, nseg, (int)(unsigned)epoch);
-
-            // table entries are fetched 32 pages at a time
-            int tbl_page0 = 0, tbl = 0;
-            for (int u = 0; ok && u < seg_len; ++u) {
-                const int page0 = first_page + (j + u) * kPagesPerStage;
-                const int np = min(kPagesPerStage, last_page + 1 - page0);
-                if ((u & (32 / kPagesPerStage - 1)) == 0) {
-                    tbl_page0 = page0;
-                    if (j + u == 0 && head_tbl_e == e) {
-                        tbl = head_tbl;           // the shard's first pages: same for every KV head
-                    } else {
-                        tbl = load_tbl(b, page0, last_page);
-                        if (j + u == 0) { head_tbl = tbl; head_tbl_e = e; }
+            while (ok && pos < pos1) {
+                while (prefix[e + 1] <= pos) ++e;  // skip empty entries
+                const int base = prefix[e];
+                const int nunits = (prefix[e + 1] - base) / Hkv;
+                const int r = pos - base;
+                const int c = r / nunits, j = r - c * nunits;
+                const int seg_len = min(nunits - j, pos1 - pos);
+                const int b = e / S;
+                if (e != cur_e) {
+                    if (e == nxt_e) clamp_range(nxt_r0, nxt_r1, nxt_len, beg, end);
+                    else clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[b], beg, end);
+                    cur_e = e;
+                    if (e == nxt_tbl_e) { head_tbl = nxt_tbl; head_tbl_e = e; }
+                    // start fetching the next non-empty shard's range; it is consumed a segment later
+                    int e2 = e + 1;
+                    while (e2 < n_entries && prefix[e2 + 1] == prefix[e2]) ++e2;
+                    nxt_e = -1;
+                    if (e2 < n_entries && prefix[e2] < pos1) {
+                        nxt_e = e2;
+                        nxt_r0 = shard_ranges[2 * e2];
+                        nxt_r1 = shard_ranges[2 * e2 + 1];
+                        nxt_len = seq_lens[e2 / S];
                     }
                 }
-                if (u == 1 && nxt_e >= 0 && nxt_tbl_e != nxt_e) {
-                    // the next shard's range has arrived by now: fetch its first table entries too
-                    int nb, ne;
-                    clamp_range(nxt_r0, nxt_r1, nxt_len, nb, ne);
-                    nxt_tbl = load_tbl(nxt_e / S, nb >> 4, (ne - 1) >> 4);
-                    nxt_tbl_e = nxt_e;
-                }
-                const int i = lane % kPagesPerStage;    // page within the stage
-                const int part = lane / kPagesPerStage; // 0: K page, 1: V page (>= 2: idle lane)
-                int phys = __shfl_sync(0xffffffffu, tbl, (page0 - tbl_page0) + i);
-                bool bad = false;
-                if (P.check_bounds && (phys < 0 || (long long)phys >= P.num_pages)) { bad = true; phys = 0; }
-                const unsigned bad_mask = __ballot_sync(0xffffffffu, bad && i < np && part == 0) & 0xffu;
-                const bool issuer = (i < np) && (part < 2);
+                const int first_page = beg >> 4, last_page = (end - 1) >> 4;
+                // the pieces that touch this unit: one segment each, slot = unit + piece (both increase along
+                // the unit space, so no two segments share a slot)
+                const int p0 = base + c * nunits;
+                const int first_piece = piece_of(pg, n_ctas, p0), last_piece = piece_of(pg, n_ctas, p0 + nunits - 1);
+                const int nseg = last_piece - first_piece + 1;
+                const int first_slot = e * Hkv + c + first_piece;
+                if (pos == piece_pos0 && lane == 0)   // does this piece start inside a unit?  (the finish kernel's input)
+                    piece_info[piece] = make_int4(j > 0 ? e * Hkv + c : -1, first_slot, nseg, (int)(unsigned)epoch);
 
-                if (pg.n_chunks > 0 && pos + u == draw_at && lane == 0) drawn = atomicAdd(header + kHdrChunk, 1ull);
-                if (!mbar_wait(smem_u32(&sm.empty_bar[stage]), phase ^ 1, abort_flag)) { ok = false; break; }
-                const bool first = (u == 0), last = (u == seg_len - 1);
-                const uint32_t full = smem_u32(&sm.full_bar[stage]);
-                if (lane == 0) {
-                    StageMeta mt;
-                    mt.entry = e; mt.kv_head = c; mt.page0 = page0; mt.npages = np;
-                    mt.tok_beg = beg; mt.tok_end = end;
-                    mt.flags = (first ? kSegFirst : 0) | (last ? kSegLast : 0) | (nseg << 8);
-                    mt.aux = (int)bad_mask;
-                    mt.slot = e * Hkv + c + piece;
-                    sm.meta[stage] = mt;
-                    mbar_arrive_expect_tx(full, (uint32_t)np * 2u * kPageBytes + (first ? (uint32_t)G * 256u : 0u));
-                    if (bad_mask) epoch_or(header + kHdrStatus, epoch, kStatusBadPage);
+                // table entries are fetched 32 pages at a time
+                int tbl_page0 = 0, tbl = 0;
+                for (int u = 0; ok && u < seg_len; ++u) {
+                    const int page0 = first_page + (j + u) * kPagesPerStage;
+                    const int np = min(kPagesPerStage, last_page + 1 - page0);
+                    if ((u & (32 / kPagesPerStage - 1)) == 0) {
+                        tbl_page0 = page0;
+                        if (j + u == 0 && head_tbl_e == e) {
+                            tbl = head_tbl;           // the shard's first pages: same for every KV head
+                        } else {
+                            tbl = load_tbl(b, page0, last_page);
+                            if (j + u == 0) { head_tbl = tbl; head_tbl_e = e; }
+                        }
+                    }
+                    if (u == 1 && nxt_e >= 0 && nxt_tbl_e != nxt_e) {
+                        // the next shard's range has arrived by now: fetch its first table entries too
+                        int nb, ne;
+                        clamp_range(nxt_r0, nxt_r1, nxt_len, nb, ne);
+                        nxt_tbl = load_tbl(nxt_e / S, nb >> 4, (ne - 1) >> 4);
+                        nxt_tbl_e = nxt_e;
+                    }
+                    const int i = lane % kPagesPerStage;    // page within the stage
+                    const int part = lane / kPagesPerStage; // 0: K page, 1: V page (>= 2: idle lane)
+                    int phys = __shfl_sync(0xffffffffu, tbl, (page0 - tbl_page0) + i);
+                    bool bad = false;
+                    if (P.check_bounds && (phys < 0 || (long long)phys >= P.num_pages)) { bad = true; phys = 0; }
+                    const unsigned bad_mask = __ballot_sync(0xffffffffu, bad && i < np && part == 0) & 0xffu;
+                    const bool issuer = (i < np) && (part < 2);
+
+                    if (pg.n_chunks > 0 && pos + u == draw_at && lane == 0) drawn = atomicAdd(header + kHdrChunk, 1ull);
+                    if (!mbar_wait(smem_u32(&sm.empty_bar[stage]), phase ^ 1, abort_flag)) { ok = false; break; }
+                    const bool first = (u == 0), last = (u == seg_len - 1);
+                    const uint32_t full = smem_u32(&sm.full_bar[stage]);
+                    if (lane == 0) {
+                        StageMeta mt;
+                        mt.entry = e; mt.kv_head = c; mt.page0 = page0; mt.npages = np;
+                        mt.tok_beg = beg; mt.tok_end = end;
+                        mt.flags = (first ? kSegFirst : 0) | (last ? kSegLast : 0) | (nseg << 8);
+                        mt.aux = (int)bad_mask;
+                        mt.slot = e * Hkv + c + piece;
+                        sm.meta[stage] = mt;
+                        mbar_arrive_expect_tx(full, (uint32_t)np * 2u * kPageBytes + (first ? (uint32_t)G * 256u : 0u));
+                        if (bad_mask) epoch_or(header + kHdrStatus, epoch, kStatusBadPage);
+                    }
+                    __syncwarp();
+                    if (issuer) {
+                        const int row = (phys * Hkv + c) * kPageSize;
+                        tma_load_page(smem_u32(&sm.kv[stage][part][i][0]), part ? &v_map : &k_map, row, full, kv_policy);
+                    }
+                    if (first && lane == 0)
+                        bulk_load_1d(smem_u32(&sm.q[stage][0]), q + ((size_t)b * Hq + (size_t)c * G) * kHeadDim,
+                                     (uint32_t)G * 256u, full);
+                    ++issued;
+                    if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
-                __syncwarp();
-                if (issuer) {
-                    const int row = (phys * Hkv + c) * kPageSize;
-                    tma_load_page(smem_u32(&sm.kv[stage][part][i][0]), part ? &v_map : &k_map, row, full, kv_policy);
-                }
-                if (first && lane == 0)
-                    bulk_load_1d(smem_u32(&sm.q[stage][0]), q + ((size_t)b * Hq + (size_t)c * G) * kHeadDim,
-                                 (uint32_t)G * 256u, full);
-                ++issued;
-                if (++stage == kStages) { stage = 0; phase ^= 1; }
+                pos += seg_len;
             }
-            pos += seg_len;
-        }
-        if (!ok || pg.n_chunks == 0) break;
-        drawn = __shfl_sync(0xffffffffu, drawn, 0);
-        if ((drawn >> 20) != (epoch & ((1ull << 44) - 1))) { ok = false; break; }   // not this launch's counter
-        const int ticket = (int)(drawn & 0xFFFFFull);
-        if (ticket >= pg.n_chunks) break;
-        piece = n_ctas + ticket;
+            if (!ok || pg.n_chunks == 0) break;
+            drawn = __shfl_sync(0xffffffffu, drawn, 0);
+            if ((drawn >> 20) != (epoch & ((1ull << 44) - 1))) { ok = false; break; }   // not this launch's counter
+            const int ticket = (int)(drawn & 0xFFFFFull);
+            if (ticket >= pg.n_chunks) break;
+            piece = n_ctas + ticket;
         }
         if (ok) {  // end-of-work marker
             if (mbar_wait(smem_u32(&sm.empty_bar[stage]), phase ^ 1, abort_flag)) {
@@ -577,7 +577,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             const size_t out_row = ((size_t)mt.entry * Hq + (size_t)mt.kv_head * G);  // + head
             float *seg_slot = seg + (size_t)mt.slot * seg_stride;
 #pragma unroll
-            for (int hr = 0; hr < G / RG; ++hr) {
+            for (int hr = 0; hr < (G + RG - 1) / RG; ++hr) {
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     const int head = 2 * t + hh;
@@ -591,11 +591,12 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                     }
                 }
                 if (!red_sync(0, red_phase0)) return;
-                {
-                    // kThreadsPerHead threads share a head: the eight warps' weights are computed once per thread
-                    constexpr int kThreadsPerHead = kConsumerThreads / RG;
-                    const int hl = tid / kThreadsPerHead, d0 = tid % kThreadsPerHead;
-                    const int head = hr * RG + hl;
+                // kThreadsPerHead threads share a head: the eight warps' weights are computed once per thread
+                // (a group size that is not a multiple of the round leaves the last round's spare threads idle)
+                constexpr int kThreadsPerHead = kConsumerThreads / RG;
+                const int hl = tid / kThreadsPerHead, d0 = tid % kThreadsPerHead;
+                const int head = hr * RG + hl;
+                if (hl < RG && head < G) {
                     float M = neg_inf();
 #pragma unroll
                     for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm.red_ml[w][head][0]);
@@ -774,7 +775,11 @@ inline int launch_sweep(const void *q, const void *k_cache, const void *v_cache,
     switch (P.group) {
     case 1: return launch_sweep_g<1>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
     case 2: return launch_sweep_g<2>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
+    case 3: return launch_sweep_g<3>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
     case 4: return launch_sweep_g<4>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
+    case 5: return launch_sweep_g<5>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
+    case 6: return launch_sweep_g<6>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
+    case 7: return launch_sweep_g<7>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
     default: return launch_sweep_g<8>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
     }
 }

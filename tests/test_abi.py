@@ -64,7 +64,7 @@ def test_workspace_bytes():
     ("num_pages", 0, qf.QF_ERR_BAD_SHAPE),
     ("head_dim", 64, qf.QF_ERR_UNSUPPORTED),
     ("page_size", 32, qf.QF_ERR_UNSUPPORTED),
-    ("num_q_heads", 24, qf.QF_ERR_UNSUPPORTED),    # group of 3
+    ("num_q_heads", 72, qf.QF_ERR_UNSUPPORTED),    # group of 9
 ])
 def test_bad_params_are_rejected_before_any_launch(field, value, code):
     p = good()

@@ -38,7 +38,7 @@ KERNELS = [pytest.param((0, 16), id="unit16"), pytest.param((0, 8), id="unit8"),
 
 # T1: every short length, both group sizes, shuffled table: tail-page masking, first-tile guard
 @pytest.mark.parametrize("flags", KERNELS)
-@pytest.mark.parametrize("G", [1, 2, 4, 8])
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 6, 7, 8])
 def test_every_short_length(G, flags):
     flags, Hkv = flags
     lens = list(range(1, 49))
@@ -220,7 +220,7 @@ def test_combine_on_handmade_states():
 
 # medium cases that span many stages, several CTA slices and ragged tails
 @pytest.mark.parametrize("flags", KERNELS)
-@pytest.mark.parametrize("G,seed", [(2, 0), (4, 1), (8, 2), (1, 3)])
+@pytest.mark.parametrize("G,seed", [(2, 0), (4, 1), (8, 2), (1, 3), (3, 4), (5, 5), (6, 6), (7, 7)])
 def test_medium_ragged_batch(G, seed, flags):
     flags, Hkv = flags
     rng = np.random.default_rng(seed)
@@ -266,6 +266,8 @@ def test_small_configs_elementwise():
     (2, 60_000, 60_000, 8, 2),    # two very long units per KV head: every unit cut many times
     (10, 20_000, 4096, 8, 4),     # ~12,600 stage units: drawing is on by default
     (5, 33_000, 7000, 2, 8),      # G = 8 (two epilogue rounds), few KV heads
+    (4, 40_000, 5000, 8, 5),      # G = 5 (Qwen3-14B's 40 / 8 heads): a second round of one head
+    (3, 30_000, 30_000, 4, 7),    # G = 7, long units cut many times
 ])
 def test_drawn_chunk_schedule(B, L, shard, Hkv, G):
     rng = np.random.default_rng(B * 1000 + L)
@@ -426,7 +428,7 @@ def test_randomized_shapes_and_ranges(seed):
     # random batch, head counts, group size, lengths, unaligned / overlapping / empty shard ranges, pool slack
     rng = np.random.default_rng(1000 + seed)
     Hkv = int(rng.choice([1, 2, 3, 4, 8, 16]))
-    G = int(rng.choice([1, 2, 4, 8]))
+    G = int(rng.integers(1, 9))
     B = int(rng.integers(1, 9))
     S = int(rng.integers(1, 7))
     lens = [int(x) for x in rng.choice([0, 1, 15, 16, 17, 127, 128, 129, 500, 3000, 20000], size=B)]
