@@ -7,7 +7,6 @@ from decimal import Decimal, getcontext
 from fractions import Fraction
 
 import numpy as np
-import pytest
 import torch
 
 from oracle import qf_oracle as orc

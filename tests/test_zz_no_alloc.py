@@ -11,7 +11,6 @@ disturbed by them.
 The file name makes pytest collect it last, so a run that stops at the first failure has
 already been through every other test.
 """
-import numpy as np
 import pytest
 import torch
 
