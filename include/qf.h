@@ -16,7 +16,10 @@
  *
  * qf_decode_partial computes one such state per (request, KV shard, query
  * head); qf_combine merges a request's shard states into the full-context
- * attention output and its log-sum-exp.
+ * attention output and its log-sum-exp.  Around them: qf_combine_self and
+ * qf_append_kv (the current token's fold and cache write, Section 2),
+ * qf_decode_step_host (one step from host buffers), qf_project_pair (the
+ * cache side's W_o / W_q projections at a layer boundary, Section 4).
  *
  * Readings fixed at this boundary where the paper is silent:
  *   - grouped-query attention: query head h reads KV head h / G, G = Hq/Hkv;
@@ -87,7 +90,7 @@ enum {
     QF_OK              = 0,
     QF_ERR_NULL        = -1, /* a required pointer is NULL                         */
     QF_ERR_BAD_SHAPE   = -2, /* non-positive size, or Hq not a multiple of Hkv     */
-    QF_ERR_UNSUPPORTED = -3, /* head_dim != 128, page_size != 16, G not in 1,2,4,8 */
+    QF_ERR_UNSUPPORTED = -3, /* head_dim != 128, page_size != 16, G not in 1..8     */
     QF_ERR_WORKSPACE   = -4, /* workspace NULL, misaligned (256 B) or too small    */
     QF_ERR_CUDA        = -5, /* a CUDA call failed; text via qf_strerror           */
     QF_ERR_DEVICE      = -6, /* device is not compute capability 10.x             */
