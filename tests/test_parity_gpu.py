@@ -291,11 +291,18 @@ def test_drawn_chunk_schedule(B, L, shard, Hkv, G):
 
 
 # T9: run-to-run determinism and canaries around the outputs
-def test_determinism_and_no_stray_writes():
+@pytest.mark.parametrize("flags", [0, qf.QF_FLAG_DRAW_ALWAYS])
+def test_determinism_and_no_stray_writes(flags):
     w = wl.config3(seed=5, batch=6, hi=12000)
-    dw = DeviceWorkload(w)
+    dw = DeviceWorkload(w, flags=flags)
     canary = 1234.5
     bufs = {}
+    # the workspace too: exactly qf_workspace_bytes, with guard bytes on both sides (the segment slots of
+    # cut units and the piece records live at its end)
+    ws_big = torch.full((dw.ws_bytes + 2 * 4096,), 0x5A, dtype=torch.uint8, device="cuda")
+    off = (-ws_big.data_ptr()) % 256 + 2048
+    dw.workspace = ws_big[off:off + dw.ws_bytes]
+    assert dw.workspace.data_ptr() % 256 == 0
     for name in ("o_part", "m_part", "lse_part", "out", "lse"):
         t = getattr(dw, name)
         big = torch.full((t.numel() + 512,), canary, dtype=torch.float32, device="cuda")
@@ -311,6 +318,7 @@ def test_determinism_and_no_stray_writes():
             assert np.array_equal(x, y)
     for name, big in bufs.items():
         assert (big[:256] == canary).all() and (big[-256:] == canary).all(), name
+    assert (ws_big[:off] == 0x5A).all() and (ws_big[off + dw.ws_bytes:] == 0x5A).all(), "write outside the workspace"
     T.compare_all(dw, w)
 
 
