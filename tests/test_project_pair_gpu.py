@@ -180,3 +180,26 @@ def test_graph_replay_with_new_inputs():
         ref_u, ref_q = orc.project_pair(a2, z, w_o, g, w_q, eps=1e-6)
         check(host_bits(u_dev), host_bits(q_dev), ref_u, ref_q, f"replay {it}")
         assert qf.project_status(args[8]) == 0
+
+
+def test_no_stray_writes():
+    # outputs and workspace sit inside guard regions; nothing outside them may change
+    batch, d_model, n_q = 17, 1024, 2048
+    a, z, w_o, g, w_q = make_inputs(batch, d_model, n_q, seed=31)
+    need = qf.project_workspace_bytes(batch, d_model, n_q)
+    guard = 4096
+    ws_big = torch.full((need + 2 * guard + 256,), 0x5A, dtype=torch.uint8, device="cuda")
+    off = (-ws_big.data_ptr()) % 256 + guard
+    ws = ws_big[off:off + need]
+    u_big = torch.full((batch * d_model + 1024,), 7.0, dtype=torch.bfloat16, device="cuda")
+    q_big = torch.full((batch * n_q + 1024,), 7.0, dtype=torch.bfloat16, device="cuda")
+    u = u_big[512:512 + batch * d_model].view(batch, d_model)
+    q = q_big[512:512 + batch * n_q].view(batch, n_q)
+    qf.project_pair(torch.from_numpy(a).cuda(), dev_bf16(z), dev_bf16(w_o), dev_bf16(g), dev_bf16(w_q), u, q, 1e-6, ws)
+    torch.cuda.synchronize()
+    assert qf.project_status(ws) == 0
+    assert (ws_big[:off] == 0x5A).all() and (ws_big[off + need:] == 0x5A).all()
+    for big, n in ((u_big, batch * d_model), (q_big, batch * n_q)):
+        assert (big[:512] == 7.0).all() and (big[512 + n:] == 7.0).all()
+    ref_u, ref_q = orc.project_pair(a, z, w_o, g, w_q, eps=1e-6)
+    check(host_bits(u.contiguous()), host_bits(q.contiguous()), ref_u, ref_q, "guarded")
