@@ -42,6 +42,7 @@
 namespace qf {
 
 constexpr int kProjThreads   = 128;   // thread t owns accumulator row t (one output feature)
+constexpr int kProjCtaThreads = 256;  // the CTA: those 128 plus four warps that only help stage the activations
 constexpr int kProjTileOut   = 128;   // output features per CTA = rows of the tensor-core tile
 constexpr int kProjSplits    = 8;     // K splits = CTAs of a cluster
 constexpr int kProjBoxK      = 64;    // bf16 per TMA box row: 128 bytes, one swizzle span
@@ -145,7 +146,7 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-// Dynamic shared memory: this header (2 KB), then a ring of weight boxes [128 rows][128 B], then n_boxes
+// Dynamic shared memory: this header (3 KB), then a ring of weight boxes [128 rows][128 B], then n_boxes
 // activation boxes [NP rows][128 B]; every box is 1,024-byte aligned.  The partial tile [NP][128] fp32
 // reuses the ring once the products are done (the host checks that it fits).
 struct ProjSmemHeader {
@@ -155,11 +156,11 @@ struct ProjSmemHeader {
     uint32_t tmem_base;
     int abort_flag;
     float ssq[kProjMaxBatch];      // stage 0: this rank's sums of squares; stage 1: 1/rms per request
-    float half_sum[kProjMaxBatch]; // stage 1 prologue
+    float part_sum[3][kProjMaxBatch];   // stage 1 prologue
     alignas(16) uint16_t gain[kProjMaxBoxes * kProjBoxK];   // stage 1: this K slice of g
 };
-constexpr int kProjHeaderBytes = 2048;
-static_assert(sizeof(ProjSmemHeader) <= kProjHeaderBytes, "header must fit its two kilobytes");
+constexpr int kProjHeaderBytes = 3072;
+static_assert(sizeof(ProjSmemHeader) <= kProjHeaderBytes, "header must fit its three kilobytes");
 constexpr int kProjWBoxBytes = kProjTileOut * 128;
 inline size_t proj_smem_bytes(int ring, int n_boxes, int np)
 {
@@ -189,13 +190,14 @@ inline ProjRing proj_ring(int n_boxes, int np)
 }
 
 template <int STAGE, int NP>
-__global__ void __launch_bounds__(kProjThreads, 1)
+__global__ void __launch_bounds__(kProjCtaThreads, 2)
 proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem_al = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     ProjSmemHeader &sm = *reinterpret_cast<ProjSmemHeader *>(smem_al);
     const int tid = threadIdx.x, warp = tid >> 5;
+    const bool is_main = tid < kProjThreads;   // the helper warps leave after the staging (they still join the cluster barriers)
     const int rank = (int)cluster_rank();                 // which eighth of K
     const int tile = (int)blockIdx.x / kProjSplits;       // which 128 output features
     const int k_slice = A.k_total / kProjSplits, n_boxes = k_slice / kProjBoxK;
@@ -249,14 +251,14 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
 #pragma unroll
     for (int i = 0; i < NP / 8; ++i) {
         const int n = ep_n0 + 8 * i;
-        zreg[i] = (STAGE == 0 && n < A.batch) ? A.z[(size_t)n * A.n_out + ep_o] : (uint16_t)0;
+        zreg[i] = (STAGE == 0 && is_main && n < A.batch) ? A.z[(size_t)n * A.n_out + ep_o] : (uint16_t)0;
     }
     if (STAGE == 0) {
-        for (int base = tid; base < n_items; base += kProjThreads * kU) {
+        for (int base = tid; base < n_items; base += kProjCtaThreads * kU) {
             float4 lo[kU], hi[kU];
 #pragma unroll
             for (int u = 0; u < kU; ++u) {
-                const int idx = base + u * kProjThreads;
+                const int idx = base + u * kProjCtaThreads;
                 if (idx < n_items) {
                     int m, k;
                     item_addr(idx, m, k);
@@ -267,7 +269,7 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
             }
 #pragma unroll
             for (int u = 0; u < kU; ++u) {
-                const int idx = base + u * kProjThreads;
+                const int idx = base + u * kProjCtaThreads;
                 if (idx < n_items) {
                     int m, k;
                     item_addr(idx, m, k);
@@ -278,13 +280,13 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
         }
     } else {
         // the gain slice and the first batch of the stream go out before the sums of squares are waited for
-        for (int i = tid; i < k_slice / 8; i += kProjThreads)
+        for (int i = tid; i < k_slice / 8; i += kProjCtaThreads)
             reinterpret_cast<uint4 *>(sm.gain)[i] = *reinterpret_cast<const uint4 *>(A.g + k0 + i * 8);
         uint4 uw[kU];
         auto load_batch = [&](int base) {
 #pragma unroll
             for (int u = 0; u < kU; ++u) {
-                const int idx = base + u * kProjThreads;
+                const int idx = base + u * kProjCtaThreads;
                 if (idx < n_items) {
                     int m, k;
                     item_addr(idx, m, k);
@@ -294,31 +296,33 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
         };
         load_batch(tid);
         {
-            // 1/rms per request from stage 0's per-tile sums of squares, summed in tile order (two interleaved halves)
-            const int n = tid & (kProjMaxBatch - 1), half = tid / kProjMaxBatch;
+            // 1/rms per request from stage 0's per-tile sums of squares: four interleaved quarters of the tiles, each
+            // summed in tile order, then added in quarter order
+            const int n = tid & (kProjMaxBatch - 1), quarter = tid / kProjMaxBatch;
             float s = 0.f;
             if (n < A.batch) {
-                for (int p0 = half; p0 < A.ssq_tiles; p0 += 2 * kU) {
+                for (int p0 = quarter; p0 < A.ssq_tiles; p0 += 4 * kU) {
                     float v[kU];
 #pragma unroll
                     for (int u = 0; u < kU; ++u) {
-                        const int p = p0 + 2 * u;
+                        const int p = p0 + 4 * u;
                         v[u] = (p < A.ssq_tiles) ? ld_sync_f32(A.ssq_part + (size_t)p * kProjMaxBatch + n) : 0.f;
                     }
 #pragma unroll
                     for (int u = 0; u < kU; ++u) s += v[u];
                 }
             }
-            if (half == 1) sm.half_sum[n] = s;
+            if (quarter > 0) sm.part_sum[quarter - 1][n] = s;
             __syncthreads();
-            if (half == 0) sm.ssq[n] = 1.0f / sqrtf((s + sm.half_sum[n]) * A.inv_d_model + A.eps);
+            if (quarter == 0)
+                sm.ssq[n] = 1.0f / sqrtf((((s + sm.part_sum[0][n]) + sm.part_sum[1][n]) + sm.part_sum[2][n]) * A.inv_d_model + A.eps);
             __syncthreads();
         }
-        for (int base = tid; base < n_items; base += kProjThreads * kU) {
+        for (int base = tid; base < n_items; base += kProjCtaThreads * kU) {
             if (base != tid) load_batch(base);
 #pragma unroll
             for (int u = 0; u < kU; ++u) {
-                const int idx = base + u * kProjThreads;
+                const int idx = base + u * kProjCtaThreads;
                 if (idx < n_items) {
                     int m, k;
                     item_addr(idx, m, k);
@@ -335,7 +339,7 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
             }
         }
     }
-    for (int idx = n_items + tid; idx < NP * chunks_per_row; idx += kProjThreads) {   // padding rows
+    for (int idx = n_items + tid; idx < NP * chunks_per_row; idx += kProjCtaThreads) {   // padding rows
         int m, k;
         item_addr(idx, m, k);
         *x_slot(m, k) = make_uint4(0u, 0u, 0u, 0u);
@@ -384,6 +388,12 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
                     if (mbar_try_wait(smem_u32(&sm.w_full[r % slots]), (uint32_t)((r / slots) & 1))) break;
             mbar_arrive(smem_u32(&sm.mma_done));
         }
+    }
+    if (!is_main) {   // helper warps: nothing left to do but keep the cluster barriers' counts whole
+        cluster_sync_all();
+        cluster_sync_all();
+        if (STAGE == 0) cluster_sync_all();
+        return;
     }
     const bool done = mbar_wait(smem_u32(&sm.mma_done), 0, abort_flag) && !*abort_flag;
     if (!done && tid == 0) { sm.abort_flag = 1; atomicOr(A.status, (unsigned)kStatusTimeout); }
@@ -539,7 +549,7 @@ cudaError_t launch_proj_np(const CUtensorMap &map, const ProjArgs &args, cudaStr
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(args.n_out / kProjTileOut * kProjSplits));
-    cfg.blockDim = dim3(kProjThreads);
+    cfg.blockDim = dim3(kProjCtaThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
