@@ -27,7 +27,7 @@
 //
 // Every wait on an mbarrier is bounded; a wait that runs out raises the CTA's abort flag and a status bit,
 // the CTA stops computing but still takes part in the cluster barriers, drains its copies and frees its
-// tensor memory.  No TMA multicast is used.
+// tensor memory.  Every TMA load lands in the shared memory of the CTA that issued it.
 #pragma once
 
 #include <cuda.h>
