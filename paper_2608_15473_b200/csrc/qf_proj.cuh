@@ -123,6 +123,12 @@ __device__ __forceinline__ float ld_peer_f32(uint32_t local_smem_addr, uint32_t 
 }
 // One request: `sb` adjacent boxes (the map's box is [sb column blocks][128 rows][64 bf16]) starting at weight
 // row `row` and column block `kblock`; they land as sb consecutive swizzled [128][128 B] tiles.
+__device__ __forceinline__ void st_peer_f32(uint32_t local_smem_addr, uint32_t rank, float v)
+{
+    uint32_t ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_smem_addr), "r"(rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(v) : "memory");
+}
 __device__ __forceinline__ void tma_load_boxes(uint32_t dst, const CUtensorMap *map, int row, int kblock, uint32_t bar,
                                                unsigned long long policy)
 {
@@ -146,7 +152,7 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-// Dynamic shared memory: this header (3 KB), then a ring of weight boxes [128 rows][128 B], then n_boxes
+// Dynamic shared memory: this header (5 KB), then a ring of weight boxes [128 rows][128 B], then n_boxes
 // activation boxes [NP rows][128 B]; every box is 1,024-byte aligned.  The partial tile [NP][128] fp32
 // reuses the ring once the products are done (the host checks that it fits).
 struct ProjSmemHeader {
@@ -157,10 +163,11 @@ struct ProjSmemHeader {
     int abort_flag;
     float ssq[kProjMaxBatch];      // stage 0: this rank's sums of squares; stage 1: 1/rms per request
     float part_sum[3][kProjMaxBatch];   // stage 1 prologue
+    float ssq_recv[kProjSplits][kProjMaxBatch];   // stage 0, rank 0: every rank's sums of squares, pushed by their owners
     alignas(16) uint16_t gain[kProjMaxBoxes * kProjBoxK];   // stage 1: this K slice of g
 };
-constexpr int kProjHeaderBytes = 3072;
-static_assert(sizeof(ProjSmemHeader) <= kProjHeaderBytes, "header must fit its three kilobytes");
+constexpr int kProjHeaderBytes = 5120;
+static_assert(sizeof(ProjSmemHeader) <= kProjHeaderBytes, "header must fit its five kilobytes");
 constexpr int kProjWBoxBytes = kProjTileOut * 128;
 inline size_t proj_smem_bytes(int ring, int n_boxes, int np)
 {
@@ -392,7 +399,6 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
     if (!is_main) {   // helper warps: nothing left to do but keep the cluster barriers' counts whole
         cluster_sync_all();
         cluster_sync_all();
-        if (STAGE == 0) cluster_sync_all();
         return;
     }
     const bool done = mbar_wait(smem_u32(&sm.mma_done), 0, abort_flag) && !*abort_flag;
@@ -449,20 +455,18 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
                 // sum of squares over the rank's 16 features: the 16 lanes of a half warp, fixed tree
 #pragma unroll
                 for (int off = 8; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
-                if (ep_j == 0) sm.ssq[n] = sq;
+                if (ep_j == 0) st_peer_f32(smem_u32(&sm.ssq_recv[rank][n]), 0u, sq);   // into rank 0's shared memory
             }
         }
     }
-    cluster_sync_all();          // partial tiles are no longer read; stage 0: every rank's sums of squares are in place
-    if (STAGE == 0) {
-        if (rank == 0 && tid < NP) {
-            float s = 0.f;
-            const uint32_t addr = smem_u32(&sm.ssq[tid]);
+    // Partial tiles are no longer read by anybody, and (stage 0) every rank's sums of squares have arrived in
+    // rank 0's shared memory: after this barrier a CTA touches only its own shared memory, so it may leave.
+    cluster_sync_all();
+    if (STAGE == 0 && rank == 0 && tid < NP) {
+        float s = 0.f;
 #pragma unroll
-            for (int c = 0; c < kProjSplits; ++c) s += ld_peer_f32(addr, (uint32_t)c);
-            A.ssq_part[(size_t)tile * kProjMaxBatch + tid] = (tid < A.batch) ? s : 0.f;
-        }
-        cluster_sync_all();      // nobody leaves while rank 0 still reads its shared memory
+        for (int c = 0; c < kProjSplits; ++c) s += sm.ssq_recv[c][tid];
+        A.ssq_part[(size_t)tile * kProjMaxBatch + tid] = (tid < A.batch) ? s : 0.f;
     }
     if (warp == 0) tmem_dealloc(tmem, 64);
 }
