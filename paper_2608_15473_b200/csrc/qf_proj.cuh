@@ -175,8 +175,9 @@ inline size_t proj_smem_bytes(int ring, int n_boxes, int np)
 }
 // The ring: `slots` requests in flight, each of `sb` adjacent boxes (sb divides the slice's box count).
 // Preferred: the largest request that still leaves room for two CTAs per SM (then every cluster of a product
-// is resident at once), with at least two slots unless one request covers the whole slice; the ring must also
-// hold the partial tile.  Falls back to one CTA per SM when nothing smaller fits.
+// is resident at once), and only then as many slots as fit: the bytes a request reads contiguously per weight
+// row matter more than the ring's depth (one 512-byte-per-row request at a time beat two 256-byte ones in
+// flight).  The ring must also hold the partial tile.  Falls back to one CTA per SM when nothing smaller fits.
 struct ProjRing { int sb, slots; };
 inline ProjRing proj_ring(int n_boxes, int np)
 {
@@ -187,7 +188,6 @@ inline ProjRing proj_ring(int n_boxes, int np)
             if (n_boxes % sb) continue;
             const int n_req = n_boxes / sb;
             for (int slots = (n_req < kProjMaxRing ? n_req : kProjMaxRing); slots >= 1; --slots) {
-                if (slots == 1 && n_req > 1) break;
                 if (sb * slots < need) break;
                 if (proj_smem_bytes(sb * slots, n_boxes, np) <= budget) return ProjRing{sb, slots};
             }
@@ -363,7 +363,16 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
         constexpr uint32_t idesc = umma_idesc_bf16(NP);
         bool ok = true;
         int consumed = 0;
-        for (int r = 0; r < n_req; ++r) {
+        for (int r = 0; r < n_req && ok; ++r) {
+            // keep the ring full: the slot of the next request to issue was last used by request (issued - slots),
+            // whose products must have completed (tcgen05.commit on the slot's barrier) before it is overwritten
+            while (issued < n_req && issued < r + slots) {
+                const int prev = issued - slots;
+                if (prev >= 0 &&
+                    !mbar_wait(smem_u32(&sm.w_empty[prev % slots]), (uint32_t)((prev / slots) & 1), abort_flag)) { ok = false; break; }
+                issue_req(issued++);
+            }
+            if (!ok) break;
             const int slot = r % slots;
             if (!mbar_wait(smem_u32(&sm.w_full[slot]), (uint32_t)((r / slots) & 1), abort_flag)) { ok = false; break; }
             consumed = r + 1;
@@ -377,12 +386,6 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
                     umma_bf16(tmem, ad + 2 * kk, bd + 2 * kk, idesc, (i | kk) ? 1u : 0u);
             }
             umma_commit(smem_u32(&sm.w_empty[slot]));     // arrives when the products above have completed
-            // refill the slot of the request before this one: its products have had this iteration to complete
-            if (r >= 1 && issued < n_req) {
-                const int ps = (r - 1) % slots;
-                if (!mbar_wait(smem_u32(&sm.w_empty[ps]), (uint32_t)(((r - 1) / slots) & 1), abort_flag)) { ok = false; break; }
-                issue_req(issued++);
-            }
         }
         if (ok) {
             umma_commit(smem_u32(&sm.mma_done));
