@@ -222,3 +222,22 @@ def test_no_stray_writes():
         assert (big[:512] == 7.0).all() and (big[512 + n:] == 7.0).all()
     ref_u, ref_q = orc.project_pair(a, z, w_o, g, w_q, eps=1e-6)
     check(host_bits(u.contiguous()), host_bits(q.contiguous()), ref_u, ref_q, "guarded")
+
+
+@pytest.mark.parametrize("seed", list(range(12)))
+def test_random_shapes(seed):
+    # every supported K (multiples of 512 up to 5,120) picks its own ring of weight requests: 1 to 10 boxes per
+    # CTA, one to four requests; batches straddle the 16-column padding steps
+    rng = np.random.default_rng(500 + seed)
+    dims = [512 * k for k in range(1, 11)]
+    for _ in range(50):
+        batch = int(rng.integers(1, 65))
+        d_model, n_q = int(rng.choice(dims)), int(rng.choice(dims))
+        if qf.project_workspace_bytes(batch, d_model, n_q) > 0:
+            break
+    else:
+        pytest.skip("no supported shape drawn")
+    a, z, w_o, g, w_q = make_inputs(batch, d_model, n_q, seed=seed)
+    u, q, _ = run_gpu(a, z, w_o, g, w_q, 1e-6)
+    ref_u, ref_q = orc.project_pair(a, z, w_o, g, w_q, eps=1e-6)
+    check(u, q, ref_u, ref_q, f"seed={seed} batch={batch} d_model={d_model} n_q={n_q}")
