@@ -173,3 +173,64 @@ def test_decode_loop_is_a_fold_over_steps():
     # the device cache equals the host mirror bit for bit
     kc = dw.k_cache.view(torch.int16).cpu().numpy().view(np.uint16)
     assert np.array_equal(kc, w.k_cache)
+
+
+def test_decode_loop_replayed_from_one_cuda_graph():
+    # One decode step (sweep, fold of the current token, cache write, length advance) captured ONCE and replayed:
+    # the lengths live on the device and grow between replays, so every replay plans a different sweep inside the
+    # kernel; the result of every step must equal attention over all positions so far plus the current one.
+    lens0 = [3, 500, 4090, 12_000]
+    steps = 12
+    Hq, Hkv = 32, 8
+    cap = [L + steps for L in lens0]
+    w = wl.make_workload("gloop", cap, [wl.fixed_shards(c, 4096) for c in cap], Hq, Hkv, seed=131)
+    w.seq_lens = np.asarray(lens0, np.int32)
+    rng = np.random.default_rng(131)
+    dw = DeviceWorkload(w)
+    dw.seq_lens.copy_(torch.from_numpy(w.seq_lens).cuda())
+    sh = T.oracle_shape(w)
+    out = torch.empty_like(dw.out)
+    lse = torch.empty_like(dw.lse)
+    k_in = torch.empty((w.batch, Hkv, 128), dtype=torch.bfloat16, device="cuda")
+    v_in = torch.empty_like(k_in)
+
+    def one_step(stream):
+        dw.sweep(stream)
+        qf.combine_self(dw.o_part, dw.lse_part, dw.shard_counts, dw.q, k_in, v_in, out, lse, dw.params, stream)
+        qf.append_kv(dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens, k_in, v_in, dw.params, stream)
+        dw.seq_lens.add_(1)
+
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        # one un-captured step first (one-time set-up), on throw-away inputs, then restore the state it changed
+        k_before, v_before = dw.k_cache.clone(), dw.v_cache.clone()
+        k_in.zero_(); v_in.zero_()
+        one_step(s)
+        torch.cuda.synchronize()
+        dw.k_cache.copy_(k_before); dw.v_cache.copy_(v_before)
+        dw.seq_lens.copy_(torch.from_numpy(w.seq_lens).cuda())
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            one_step(s)
+    # the capture did not run anything: lengths are still the initial ones
+    assert np.array_equal(dw.seq_lens.cpu().numpy(), w.seq_lens)
+    for j in range(steps):
+        qj = wl.f32_to_bf16_bits(rng.standard_normal(w.q.shape).astype(np.float32))
+        kj = wl.f32_to_bf16_bits(rng.standard_normal((w.batch, Hkv, 128)).astype(np.float32))
+        vj = wl.f32_to_bf16_bits(rng.standard_normal((w.batch, Hkv, 128)).astype(np.float32))
+        dw.q.copy_(dev_bf16(qj)); k_in.copy_(dev_bf16(kj)); v_in.copy_(dev_bf16(vj))
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        for b in range(w.batch):
+            L = int(w.seq_lens[b])
+            w.k_cache[w.block_table[b, L // 16], :, L % 16] = kj[b]
+            w.v_cache[w.block_table[b, L // 16], :, L % 16] = vj[b]
+        w.seq_lens = w.seq_lens + 1
+        w.q = qj
+        assert np.array_equal(dw.seq_lens.cpu().numpy(), w.seq_lens)
+        ref_out, ref_lse = orc.decode_full(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, sh)
+        assert T.out_err(out.cpu().numpy(), ref_out) <= T.ENG_OUT, j
+        assert T.lse_err(lse.cpu().numpy(), ref_lse) <= T.ENG_LSE, j
+        assert dw.status() == 0
