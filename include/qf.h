@@ -124,6 +124,9 @@ typedef struct qf_params {
     int32_t flags;             /* QF_FLAG_*                                      */
     int64_t num_pages;         /* pages in k_cache / v_cache                     */
     float   sm_scale;          /* <= 0 means 1/sqrt(head_dim)                    */
+    int32_t out_shards;        /* qf_decode_partial only: shard slots per request of
+                                  the OUTPUT arrays (0 = max_shards)             */
+    int32_t out_shard_offset;  /* ... and the slot this call's shard 0 goes to    */
     int32_t reserved;          /* set to 0                                       */
 } qf_params;
 
@@ -152,6 +155,12 @@ size_t qf_workspace_bytes(const qf_params *p);
  *     o_part[b,s,h,:] = O(S),  m_part[b,s,h] = max_i s_i,
  *     lse_part[b,s,h] = log Z(S).
  * Every one of the B*S slots is written (empty: 0, -inf, -inf).
+ * With out_shards > 0 the outputs are laid out for a larger shard table,
+ * o_part [B, out_shards, Hq, D] and m_part / lse_part [B, out_shards, Hq], and
+ * this call writes slots out_shard_offset .. out_shard_offset + S - 1 of every
+ * request and nothing else (Section 5: a request's cache split over devices;
+ * each device sweeps the shards it holds straight into the merging device's
+ * arrays, which may be peer memory: the sweep writes states with plain stores).
  * All pointers are device pointers; block_table may be NULL (identity).
  * K/V pool pointers must be 128-byte aligned.  Enqueues on cuda_stream: the
  * sweep kernel, then a small finish kernel that merges the (shard, KV head)

@@ -55,6 +55,8 @@ class QFParams(ctypes.Structure):
         ("flags", ctypes.c_int32),
         ("num_pages", ctypes.c_int64),
         ("sm_scale", ctypes.c_float),
+        ("out_shards", ctypes.c_int32),
+        ("out_shard_offset", ctypes.c_int32),
         ("reserved", ctypes.c_int32),
     ]
 
@@ -142,9 +144,9 @@ def _stream(stream) -> Optional[int]:
 
 def params(batch: int, num_q_heads: int, num_kv_heads: int, max_pages_per_req: int, max_shards: int,
            num_pages: int, head_dim: int = 128, page_size: int = 16, flags: int = 0,
-           sm_scale: float = 0.0) -> QFParams:
+           sm_scale: float = 0.0, out_shards: int = 0, out_shard_offset: int = 0) -> QFParams:
     return QFParams(batch, num_q_heads, num_kv_heads, head_dim, page_size, max_pages_per_req, max_shards,
-                    flags, num_pages, sm_scale, 0)
+                    flags, num_pages, sm_scale, out_shards, out_shard_offset, 0)
 
 
 def version() -> int:

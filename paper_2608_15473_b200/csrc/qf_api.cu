@@ -33,6 +33,9 @@ int validate(const qf_params *p)
         p->max_shards <= 0 || p->num_pages <= 0 || p->head_dim <= 0 || p->page_size <= 0)
         return QF_ERR_BAD_SHAPE;
     if (p->num_q_heads % p->num_kv_heads) return QF_ERR_BAD_SHAPE;
+    if (p->out_shards < 0 || p->out_shard_offset < 0) return QF_ERR_BAD_SHAPE;
+    if (p->out_shards > 0 && (long long)p->out_shard_offset + p->max_shards > p->out_shards) return QF_ERR_BAD_SHAPE;
+    if (p->out_shards == 0 && p->out_shard_offset != 0) return QF_ERR_BAD_SHAPE;
     if (p->head_dim != qf::kHeadDim || p->page_size != qf::kPageSize) return QF_ERR_UNSUPPORTED;
     const int G = p->num_q_heads / p->num_kv_heads;
     if (G < 1 || G > 8) return QF_ERR_UNSUPPORTED;
@@ -52,6 +55,8 @@ qf::DevParams dev_params(const qf_params *p)
     d.group = p->num_q_heads / p->num_kv_heads;
     d.max_pages_per_req = p->max_pages_per_req;
     d.max_shards = p->max_shards;
+    d.out_shards = p->out_shards > 0 ? p->out_shards : p->max_shards;
+    d.out_shard0 = p->out_shards > 0 ? p->out_shard_offset : 0;
     d.check_bounds = (p->flags & QF_FLAG_CHECK_BOUNDS) ? 1 : 0;
     d.draw_always = (p->flags & QF_FLAG_DRAW_ALWAYS) ? 1 : 0;
     d.num_pages = p->num_pages;
@@ -294,6 +299,7 @@ int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_c
     if (rc != QF_OK) return rc;
     if (!q_host || !k_cache || !v_cache || !seq_lens_host || !shard_ranges_host || !out_host || !lse_host)
         return QF_ERR_NULL;
+    if (p->out_shards != 0) return QF_ERR_BAD_SHAPE;   // the step owns its own shard-state arrays
     const StepLayout L = step_layout(p);
     if (!dev_scratch || ((uintptr_t)dev_scratch & 255) || dev_scratch_bytes < L.total) return QF_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;

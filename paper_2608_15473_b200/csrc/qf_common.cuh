@@ -23,6 +23,8 @@ struct DevParams {
     int group;               // G = Hq / Hkv
     int max_pages_per_req;
     int max_shards;
+    int out_shards;          // shard slots per request of the output arrays (>= out_shard0 + max_shards)
+    int out_shard0;          // output slot of this call's shard 0
     int check_bounds;
     int draw_always;         // cut the tail into drawn chunks however short the sweep is
     long long num_pages;
@@ -151,6 +153,15 @@ __device__ __forceinline__ void launch_done(unsigned long long *header, unsigned
 {
     if (epoch_arrive_crowd(header + kHdrDone, epoch) == n_ctas)
         atomicAdd(header + kHdrLaunchCount, 1ull);
+}
+
+// Row of the output arrays for entry e = b*S + s of this call: the outputs may be laid out for a larger
+// shard table (a request's cache split over devices: every device writes its own slots of the merging
+// device's arrays).
+__device__ __forceinline__ size_t out_entry(const DevParams &P, int e)
+{
+    const int b = e / P.max_shards, s = e - b * P.max_shards;
+    return (size_t)b * P.out_shards + P.out_shard0 + s;
 }
 
 // Clamp a shard's token range to the request's cached length.

@@ -72,7 +72,7 @@ finish_kernel(const int4 *__restrict__ piece_info, const unsigned long long *__r
               int max_pieces, unsigned long long *__restrict__ counters, float *__restrict__ seg, int seg_stride,
               int seg_slots,
               float *__restrict__ o_part, float *__restrict__ m_part, float *__restrict__ lse_part, int n_units,
-              int Hkv, int Hq)
+              DevParams P)
 {
     static_assert(kFinThreads >= 8 * 2 * G, "one (M, z) word per thread and batch");
     __shared__ float s_mz[8][2 * G];
@@ -92,7 +92,8 @@ finish_kernel(const int4 *__restrict__ piece_info, const unsigned long long *__r
     if (k != 1 && (k % kFinGroup) != 0) return;
     const int group = k / kFinGroup, n_groups = (nseg + kFinGroup - 1) / kFinGroup;
     const int seg0 = group * kFinGroup;
-    const size_t out_row = (size_t)(unit / Hkv) * Hq + (size_t)(unit % Hkv) * G;
+    const int Hkv = P.num_kv_heads, Hq = P.num_q_heads;
+    const size_t out_row = out_entry(P, unit / Hkv) * Hq + (size_t)(unit % Hkv) * G;
     const float kLn2 = 0.6931471805599453f;
 
     float acc[G], M[G], z[G];

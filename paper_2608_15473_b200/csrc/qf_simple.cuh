@@ -96,7 +96,7 @@ sweep_simple_kernel(const uint16_t *__restrict__ q, const uint16_t *__restrict__
         float M = neg_inf();
 #pragma unroll
         for (int w = 0; w < kSimpleWarps; ++w) M = fmaxf(M, sm_m[w][g]);
-        const size_t slot = ((size_t)b * S + s) * Hq + c * G + g;
+        const size_t slot = out_entry(P, b * S + s) * Hq + c * G + g;
         if (M == neg_inf()) {  // empty shard
             o_part[slot * kHeadDim + d] = 0.f;
             if (d == 0) { m_part[slot] = neg_inf(); lse_part[slot] = neg_inf(); }

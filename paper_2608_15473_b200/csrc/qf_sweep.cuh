@@ -496,11 +496,12 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     // empty shards: (0, -inf, -inf), spread over all CTAs' consumer warps while the ring fills
     for (int e = (int)blockIdx.x * kConsumerWarps + warp; e < n_entries; e += (int)gridDim.x * kConsumerWarps) {
         if (prefix[e + 1] != prefix[e]) continue;
-        float4 *o4 = reinterpret_cast<float4 *>(o_part + (size_t)e * Hq * kHeadDim);
+        const size_t oe = out_entry(P, e);
+        float4 *o4 = reinterpret_cast<float4 *>(o_part + oe * Hq * kHeadDim);
         for (int i = lane; i < Hq * (kHeadDim / 4); i += 32) o4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int h = lane; h < Hq; h += 32) {
-            m_part[(size_t)e * Hq + h] = neg_inf();
-            lse_part[(size_t)e * Hq + h] = neg_inf();
+            m_part[oe * Hq + h] = neg_inf();
+            lse_part[oe * Hq + h] = neg_inf();
         }
     }
 
@@ -574,7 +575,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             }
             constexpr int RG = SweepSmem<G>::kRoundHeads;
             const int nseg = mt.flags >> 8;
-            const size_t out_row = ((size_t)mt.entry * Hq + (size_t)mt.kv_head * G);  // + head
+            const size_t out_row = out_entry(P, mt.entry) * Hq + (size_t)mt.kv_head * G;  // + head
             float *seg_slot = seg + (size_t)mt.slot * seg_stride;
 #pragma unroll
             for (int hr = 0; hr < (G + RG - 1) / RG; ++hr) {
@@ -757,7 +758,7 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
     e = launch_pdl(finish_kernel<G>, dim3(n_ctas + kMaxDynChunks - 1), dim3(kFinThreads), 0, st,
                    (const int4 *)piece_info, (const unsigned long long *)header, kMaxSweepCtas + kMaxDynChunks,
                    counters, seg, wsl.seg_stride,
-                   (int)wsl.seg_slots, o, m, l, n_entries * P.num_kv_heads, P.num_kv_heads, P.num_q_heads);
+                   (int)wsl.seg_slots, o, m, l, n_entries * P.num_kv_heads, P);
     if (e != cudaSuccess) { snprintf(msg, msg_len, "finish_kernel launch: %s", cudaGetErrorString(e)); return -5; }
     *launches += 1;
     return 0;

@@ -34,9 +34,10 @@ def whole_job_throughput(total_bytes: float, max_ms_per_step: float) -> float:
 # One request's cache split over devices (Section 5): every device sweeps the shards it holds and
 # returns (O, log Z) per shard; the owner merges.  The states are tiny (one "j-th" of the sweep's
 # bytes), so the exchange is a gather of [B, S_local, Hq, D] + [B, S_local, Hq] per rank.  On GPUs
-# the same exchange needs no collective at all if o_part / lse_part passed to qf_decode_partial are
-# peer-mapped pointers into the owner's buffers: the sweep kernel writes shard states with plain
-# stores, so its epilogue is the transfer ("parked, not pushed").
+# the same exchange needs no collective at all: with out_shards / out_shard_offset in the parameters
+# (rank_sweep_params) every rank's qf_decode_partial writes its slots of the OWNER's [B, S, Hq, D] arrays,
+# passed as peer-mapped pointers; the sweep kernel writes shard states with plain stores, so its epilogue
+# is the transfer ("parked, not pushed"), and the owner merges after a barrier.
 # --------------------------------------------------------------------------------------------------
 def shard_slice(max_shards: int, world_size: int, rank: int) -> range:
     """Shard slots [lo, hi) of every request that ``rank`` sweeps: equal blocks of ceil(S/world)."""
@@ -53,6 +54,20 @@ def local_shard_ranges(shard_ranges, max_shards: int, world_size: int, rank: int
     out = torch.zeros((shard_ranges.shape[0], per, 2), dtype=shard_ranges.dtype, device=shard_ranges.device)
     out[:, :len(sl)] = shard_ranges[:, sl.start:sl.stop]
     return out
+
+
+def rank_sweep_params(p, world_size: int, rank: int):
+    """Parameters of ``rank``'s sweep when every rank writes its shard states straight into the merging device's
+    arrays (no gather): the rank sweeps S_local = ceil(S/world) slots (``local_shard_ranges``) and places them at
+    slots [rank * S_local, (rank + 1) * S_local) of arrays laid out for world * S_local slots per request.
+    The merging device then calls qf_combine with max_shards = world * S_local (padded slots are empty)."""
+    import copy
+    per = -(-int(p.max_shards) // world_size)
+    q = copy.copy(p)
+    q.max_shards = per
+    q.out_shards = per * world_size
+    q.out_shard_offset = rank * per
+    return q
 
 
 def gather_shard_states(o_local: torch.Tensor, lse_local: torch.Tensor, max_shards: int, dist):

@@ -44,8 +44,9 @@ def good():
 
 
 def test_struct_layout_matches_header():
-    assert ctypes.sizeof(qf.QFParams) == 48
+    assert ctypes.sizeof(qf.QFParams) == 56
     assert qf.QFParams.num_pages.offset == 32 and qf.QFParams.sm_scale.offset == 40
+    assert qf.QFParams.out_shards.offset == 44 and qf.QFParams.out_shard_offset.offset == 48
 
 
 def test_workspace_bytes():
@@ -65,6 +66,9 @@ def test_workspace_bytes():
     ("head_dim", 64, qf.QF_ERR_UNSUPPORTED),
     ("page_size", 32, qf.QF_ERR_UNSUPPORTED),
     ("num_q_heads", 72, qf.QF_ERR_UNSUPPORTED),    # group of 9
+    ("out_shards", 1, qf.QF_ERR_BAD_SHAPE),        # output table smaller than this call's two shards
+    ("out_shard_offset", 1, qf.QF_ERR_BAD_SHAPE),  # an offset without an output table
+    ("out_shards", -1, qf.QF_ERR_BAD_SHAPE),
 ])
 def test_bad_params_are_rejected_before_any_launch(field, value, code):
     p = good()

@@ -113,3 +113,19 @@ def test_request_split_over_two_ranks_merges_to_the_unsplit_result(tmp_path):
     mp.spawn(_sharded_rank, args=(world, port, str(tmp_path)), nprocs=world, join=True)
     err = np.load(tmp_path / "err.npy")
     assert err[0] < 1e-13 and err[1] < 1e-12 and err[2] == 1.0 and err[3] == 1.0 and err[4] == 1.0
+
+
+def test_rank_sweep_params_tile_the_owners_shard_table():
+    from paper_2608_15473_b200 import binding as qf
+    from paper_2608_15473_b200 import multi
+    p = qf.params(batch=3, num_q_heads=16, num_kv_heads=8, max_pages_per_req=64, max_shards=9, num_pages=512)
+    for world in (1, 2, 3, 4, 9, 16):
+        per = -(-9 // world)
+        covered = []
+        for rank in range(world):
+            q = multi.rank_sweep_params(p, world, rank)
+            assert (q.max_shards, q.out_shards, q.out_shard_offset) == (per, per * world, rank * per)
+            assert q.batch == p.batch and q.num_pages == p.num_pages and p.out_shards == 0   # the original is untouched
+            covered += list(range(q.out_shard_offset, q.out_shard_offset + q.max_shards))
+            assert len(multi.shard_slice(9, world, rank)) <= per
+        assert covered == list(range(per * world))

@@ -460,3 +460,58 @@ def test_randomized_shapes_and_ranges(seed):
     dw = run(w, flags)
     T.compare_all(dw, w, tag=f"seed={seed} Hkv={Hkv} G={G} B={B} S={S} flags={flags}")
     assert dw.status() == 0
+
+
+# Section 5, one request's cache split over devices, without a gather: every (virtual) rank sweeps the shard slots
+# it holds and writes them straight into the merging device's shard-state arrays (out_shards / out_shard_offset);
+# the merging device combines.  The ranks here are successive calls on one GPU, each with its own workspace, as
+# they would be separate GPUs writing through peer-mapped pointers.
+@pytest.mark.parametrize("world", [2, 3, 4])
+@pytest.mark.parametrize("flags", [0, qf.QF_FLAG_DRAW_ALWAYS, qf.QF_FLAG_SIMPLE_KERNEL])
+def test_split_request_written_in_place_by_virtual_ranks(world, flags):
+    from paper_2608_15473_b200 import multi
+    lens = [40_000, 7_000, 0, 129]
+    S = 9
+    w = wl.make_workload("split", lens, [wl.even_shards(L, S) for L in lens], 16, 8, seed=43 + world)
+    base = DeviceWorkload(w, flags=flags)
+    per = -(-S // world)
+    St = per * world
+    B, Hq = w.batch, w.num_q_heads
+    canary = 777.0
+    o_all = torch.full((B, St, Hq, 128), canary, dtype=torch.float32, device="cuda")
+    m_all = torch.full((B, St, Hq), canary, dtype=torch.float32, device="cuda")
+    l_all = torch.full((B, St, Hq), canary, dtype=torch.float32, device="cuda")
+    for rank in range(world):
+        p = multi.rank_sweep_params(base.params, world, rank)
+        ranges = multi.local_shard_ranges(base.shard_ranges, S, world, rank).contiguous()
+        ws = torch.empty(qf.workspace_bytes(p), dtype=torch.uint8, device="cuda")
+        # before the call the rank's slots still hold the canary; after it, only they have changed
+        before = o_all.clone()
+        qf.decode_partial(base.q, base.k_cache, base.v_cache, base.block_table, base.seq_lens, ranges, o_all, m_all,
+                          l_all, p, ws, ws.numel())
+        torch.cuda.synchronize()
+        lo, hi = rank * per, (rank + 1) * per
+        assert (o_all[:, lo:hi] != canary).any() and not (l_all[:, lo:hi] == canary).any()
+        untouched = torch.ones(St, dtype=torch.bool, device="cuda")
+        untouched[lo:hi] = False
+        assert torch.equal(o_all[:, untouched], before[:, untouched])
+    # the merging device: n-way combine over the padded shard table
+    out = torch.empty((B, Hq, 128), dtype=torch.float32, device="cuda")
+    lse = torch.empty((B, Hq), dtype=torch.float32, device="cuda")
+    pc = qf.params(batch=B, num_q_heads=Hq, num_kv_heads=w.num_kv_heads, max_pages_per_req=w.max_pages_per_req,
+                   max_shards=St, num_pages=w.num_pages)
+    qf.combine(o_all, l_all, None, out, lse, pc)
+    torch.cuda.synchronize()
+    sh = T.oracle_shape(w)
+    ref_out, ref_lse = orc.decode_full(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, sh)
+    assert T.out_err(out.cpu().numpy(), ref_out) <= T.ENG_OUT
+    assert T.lse_err(lse.cpu().numpy(), ref_lse) <= T.ENG_LSE
+    # and every real slot equals the oracle's shard state; padded slots are empty
+    ref_o, ref_m, ref_l = orc.decode_partial(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.shard_ranges, sh)
+    got_o, got_l = o_all.cpu().numpy().astype(np.float64), l_all.cpu().numpy().astype(np.float64)
+    for rank in range(world):
+        sl = multi.shard_slice(S, world, rank)
+        dst = slice(rank * per, rank * per + len(sl))
+        assert T.out_err(got_o[:, dst], ref_o[:, sl.start:sl.stop]) <= T.ENG_OUT
+        assert T.lse_err(got_l[:, dst], ref_l[:, sl.start:sl.stop]) <= T.ENG_LSE
+        assert np.isneginf(got_l[:, rank * per + len(sl):(rank + 1) * per]).all()
