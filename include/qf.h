@@ -56,7 +56,7 @@
  * Ownership: every pointer is borrowed for the duration of the enqueued work;
  * the library allocates no device memory, keeps no pointer after the work
  * completes and has no mutable global state beyond one-time per-device kernel
- * attributes and a small host-side cache of TMA descriptors keyed by
+ * attributes and a host-side cache of TMA descriptors (1,024 entries) keyed by
  * (pointer, num_pages, num_kv_heads).  `p` is host memory, read before return.
  *
  * Asynchrony: every call only enqueues work on `cuda_stream` (a cudaStream_t

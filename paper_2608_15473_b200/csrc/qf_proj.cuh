@@ -485,14 +485,21 @@ inline int make_weight_map(CUtensorMap *out, const void *w, int rows, int cols, 
     static EncodeFn encode = nullptr;
     static std::mutex mu;
     struct Entry { const void *w; int rows, cols, sb; CUtensorMap map; };
-    static Entry cache[32];
-    static int n_cached = 0, next = 0;
+    // One descriptor per (pointer, shape, request size), hashed by the pointer: a decode loop walks every layer's
+    // weights each step, so the cache holds a whole model's worth and a lookup is a handful of probes.
+    constexpr int kCacheEntries = 1024, kProbes = 8;
+    static Entry cache[kCacheEntries];   // zero-initialised: w == nullptr marks a free entry
+    const size_t home = (size_t)(((uintptr_t)w >> 8) * 0x9E3779B97F4A7C15ull >> 40) % kCacheEntries;
     std::lock_guard<std::mutex> lock(mu);
-    for (int i = 0; i < n_cached; ++i)
-        if (cache[i].w == w && cache[i].rows == rows && cache[i].cols == cols && cache[i].sb == sb) {
-            *out = cache[i].map;
+    size_t victim = home;
+    for (int i = 0; i < kProbes; ++i) {
+        Entry &c = cache[(home + i) % kCacheEntries];
+        if (c.w == w && c.rows == rows && c.cols == cols && c.sb == sb) {
+            *out = c.map;
             return 0;
         }
+        if (c.w == nullptr) { victim = (home + i) % kCacheEntries; break; }
+    }
     if (!encode) {
         void *fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -515,10 +522,8 @@ inline int make_weight_map(CUtensorMap *out, const void *w, int rows, int cols, 
         snprintf(msg, msg_len, "cuTensorMapEncodeTiled (weight) failed with CUresult %d", (int)r);
         return -1;
     }
-    Entry &slot = cache[next];
+    Entry &slot = cache[victim];   // a free entry among the probes, else the home entry is replaced
     slot.w = w; slot.rows = rows; slot.cols = cols; slot.sb = sb; slot.map = map;
-    next = (next + 1) % 32;
-    if (n_cached < 32) ++n_cached;
     *out = map;
     return 0;
 }

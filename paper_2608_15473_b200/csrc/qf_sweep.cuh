@@ -668,15 +668,21 @@ inline int make_pool_map(CUtensorMap *out, const void *pool, long long num_pages
     static EncodeTiledFn encode = nullptr;
     static std::mutex mu;
     struct Entry { const void *pool; long long pages; int heads; int rows; CUtensorMap map; };
-    static Entry cache[16];
-    static int n_cached = 0, next = 0;
+    // One descriptor per (pointer, shape), hashed by the pointer: a decode loop walks every layer's pools each
+    // step, so the cache holds a whole model's worth and a lookup is a handful of probes, not a scan.
+    constexpr int kCacheEntries = 1024, kProbes = 8;
+    static Entry cache[kCacheEntries];   // zero-initialised: pool == nullptr marks a free entry
+    const size_t home = (size_t)(((uintptr_t)pool >> 8) * 0x9E3779B97F4A7C15ull >> 40) % kCacheEntries;
     std::lock_guard<std::mutex> lock(mu);
-    for (int i = 0; i < n_cached; ++i)
-        if (cache[i].pool == pool && cache[i].pages == num_pages && cache[i].heads == num_kv_heads &&
-            cache[i].rows == box_rows) {
-            *out = cache[i].map;
+    size_t victim = home;
+    for (int i = 0; i < kProbes; ++i) {
+        Entry &c = cache[(home + i) % kCacheEntries];
+        if (c.pool == pool && c.pages == num_pages && c.heads == num_kv_heads && c.rows == box_rows) {
+            *out = c.map;
             return 0;
         }
+        if (c.pool == nullptr) { victim = (home + i) % kCacheEntries; break; }
+    }
     if (!encode) {
         void *fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -701,10 +707,8 @@ inline int make_pool_map(CUtensorMap *out, const void *pool, long long num_pages
         snprintf(msg, msg_len, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
         return -1;
     }
-    Entry &slot = cache[next];
+    Entry &slot = cache[victim];   // a free entry among the probes, else the home entry is replaced
     slot.pool = pool; slot.pages = num_pages; slot.heads = num_kv_heads; slot.rows = box_rows; slot.map = map;
-    next = (next + 1) % 16;
-    if (n_cached < 16) ++n_cached;
     *out = map;
     return 0;
 }
