@@ -9,17 +9,19 @@
 //   * Y^T[out x batch] = W[out x K] . X^T[K x batch]: the weight is the M-side operand of
 //     tcgen05.mma (128 output features per CTA), the batch is the N side (16..64 columns), the
 //     accumulator lives in tensor memory.
-//   * K is split eight ways over a thread-block cluster, so a 2,560 x 4,096 weight keeps 160 CTAs busy;
-//     a CTA's weight slice (128 x K/8 bf16) streams through a small ring of TMA requests, each of several
-//     adjacent 128-row x 128-byte boxes (so that a request reads 256 bytes to 1 KB contiguous per weight row:
-//     with one 128-byte box per request every row segment opened its own DRAM page and the stream ran at
-//     a third of the HBM rate); the ring's first fill is requested at the very start of the kernel, before the programmatic dependency on the
-//     previous kernel is waited for (weights are never produced on the path); a slot is refilled as soon
-//     as the products that read it have completed (tcgen05.commit on the slot's barrier).  The ring, not
-//     the whole slice, is resident so that two CTAs fit an SM and every cluster of a product is resident
+//   * K is split eight ways over a thread-block cluster, so a 2,560 x 4,096 weight keeps 160 CTAs busy.
+//     A CTA's weight slice (128 x K/8 bf16) arrives in TMA requests of several adjacent 128-row x 128-byte
+//     boxes.  How many bytes a request reads contiguously per weight row decides what the stream reaches
+//     (one 128-byte box per request: a third of the HBM rate; 512 bytes per row: more than twice that),
+//     so a request is as large as shared memory allows and the ring is as deep as what is left (often one
+//     slot).  The first requests go out at the very start of the kernel, before the programmatic dependency
+//     on the previous kernel is waited for (weights are never produced on the path); a slot is refilled as
+//     soon as the products that read it have completed (tcgen05.commit on the slot's barrier).  The ring,
+//     not the whole slice, is resident so that two CTAs fit an SM and every cluster of a product is resident
 //     at once: with the whole slice resident the kernel ran in two waves and took twice as long.
+//   * 256 threads stage the activation slice (the 128 that own accumulator rows plus four helper warps).
 //   * the eight partial tiles are summed over distributed shared memory in rank order (bit-deterministic),
-//     each rank finishing 16 of the tile's 128 output features.
+//     each rank finishing 16 of the tile's 128 output features; two cluster barriers in all.
 //
 // Stage 0 (W_o): X = bf16(a), epilogue u' = bf16(z + Y), plus each tile's sum of squares of the rounded
 // stream per request.  Stage 1 (W_q): X = bf16(g u' / sqrt(mean u'^2 + eps)) built in the prologue from
@@ -47,7 +49,7 @@ constexpr int kProjTileOut   = 128;   // output features per CTA = rows of the t
 constexpr int kProjSplits    = 8;     // K splits = CTAs of a cluster
 constexpr int kProjBoxK      = 64;    // bf16 per TMA box row: 128 bytes, one swizzle span
 constexpr int kProjMaxBoxes  = 10;    // K / 8 / 64 <= 10, i.e. K <= 5,120
-constexpr int kProjMaxRing   = 4;     // weight boxes in flight per CTA
+constexpr int kProjMaxRing   = 4;     // weight requests in flight per CTA, at most
 constexpr int kProjMaxBatch  = 64;
 constexpr int kProjRowsPerRank = kProjTileOut / kProjSplits;   // 16
 
