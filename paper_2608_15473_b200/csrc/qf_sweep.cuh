@@ -66,7 +66,7 @@ constexpr int kDynMinChunk      = QF_DYN_MIN_CHUNK;   // stage units
 #endif
 constexpr int kDynRounds        = QF_DYN_ROUNDS;      // chunk sizes halve from round to round
 constexpr int kMaxDynChunks     = kDynRounds * kMaxSweepCtas;   // bounds the segment slots
-constexpr int kDynMinUnitsPerCta = 64;                // shorter sweeps stay fully static
+constexpr int kDynMinUnitsPerCta = 112;               // shorter sweeps (under ~150 us) stay fully static: measured break-even
 static_assert(kMaxSweepCtas + kMaxDynChunks < (1 << kEpochShift), "segments of one unit must fit the arrival count");
 
 struct WorkspaceLayout {

@@ -264,7 +264,7 @@ def test_small_configs_elementwise():
     (40, 700, 130, 8, 2),         # units of one or two stages: most chunks hold several whole units
     (6, 9000, 1024, 8, 4),        # units of 8 stages
     (2, 60_000, 60_000, 8, 2),    # two very long units per KV head: every unit cut many times
-    (10, 20_000, 4096, 8, 4),     # ~12,600 stage units: drawing is on by default
+    (22, 20_000, 4096, 8, 4),     # ~21,000 stage units: drawing is on by default (from 112 per SM)
     (5, 33_000, 7000, 2, 8),      # G = 8 (two epilogue rounds), few KV heads
     (4, 40_000, 5000, 8, 5),      # G = 5 (Qwen3-14B's 40 / 8 heads): a second round of one head
     (3, 30_000, 30_000, 4, 7),    # G = 7, long units cut many times

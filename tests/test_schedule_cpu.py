@@ -33,21 +33,21 @@ def check_tiling(pieces, total, n_ctas):
 @pytest.mark.parametrize("n_ctas", [1, 2, 7, 132, 148, 160])
 def test_pieces_tile_the_unit_space_for_every_total(n_ctas):
     rng = np.random.default_rng(n_ctas)
-    totals = list(range(0, 3 * n_ctas + 3)) + [64 * n_ctas - 1, 64 * n_ctas, 64 * n_ctas + 1] + \
+    totals = list(range(0, 3 * n_ctas + 3)) + [112 * n_ctas - 1, 112 * n_ctas, 112 * n_ctas + 1] + \
         [int(x) for x in rng.integers(1, 3_000_000, size=60)] + [2**31 - 1 - 160]
     for total in totals:
         for always in (False, True):
             pieces = qf.plan_pieces(total, n_ctas, always)
             check_tiling(pieces, total, n_ctas)
             drawn = pieces[n_ctas:]
-            if total < (2 if always else 64) * n_ctas:
+            if total < (2 if always else 112) * n_ctas:
                 assert not drawn, "short sweeps stay static"
             assert len(drawn) <= 3 * 160
 
 
 def test_drawn_share_and_halving_rounds():
     n = 148
-    for total in (64 * n, 30_916, 65_536, 131_171, 1_000_003):
+    for total in (112 * n, 30_916, 65_536, 131_171, 1_000_003):
         pieces = qf.plan_pieces(total, n)
         static, drawn = pieces[:n], pieces[n:]
         static_end = static[-1][1]
