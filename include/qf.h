@@ -235,7 +235,7 @@ int qf_append_kv(void *k_cache, void *v_cache, const int32_t *block_table, const
  *   128-byte aligned.  workspace: qf_project_workspace_bytes bytes, 256-byte
  *   aligned, contents need not be initialised.
  * Supported: 1 <= batch <= 64; d_model and n_q multiples of 512, at most
- * 5,120 (for batch > 32: at least 1,024); else
+ * 5,120; else
  * QF_ERR_UNSUPPORTED (qf_project_workspace_bytes returns 0).  Larger batches
  * are run in slices of 64 by the caller.  Enqueues two kernels on cuda_stream
  * (capturable in a CUDA graph; the first call for a shape sets kernel

@@ -64,6 +64,7 @@ struct ProjArgs {
     int batch, n_out, k_total;
     int ssq_tiles;             // stage 1: number of stage 0 tiles
     int ring_sb, ring_slots;   // boxes per TMA request, requests in flight per CTA (proj_ring)
+    int recv_aliased;          // the split-K receive area reuses the ring (large batches) instead of its own room
     float inv_d_model, eps;    // stage 1
 };
 
@@ -104,33 +105,31 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
 #pragma unroll
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ void cluster_sync_all()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t cluster_rank()
 {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
-__device__ __forceinline__ float ld_peer_f32(uint32_t local_smem_addr, uint32_t rank)
+// The address, in the cluster's shared window, of CTA `rank`'s copy of one of this CTA's shared-memory locations.
+__device__ __forceinline__ uint32_t peer_addr(uint32_t local_smem_addr, uint32_t rank)
 {
     uint32_t ra;
-    float v;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_smem_addr), "r"(rank));
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
-    return v;
+    return ra;
+}
+// Store into a peer's shared memory that counts its four bytes on a transaction barrier of that same peer: the
+// receiver learns that the data has landed from its own barrier, without a cluster-wide release and acquire.
+__device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float v, uint32_t cluster_mbar)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];"
+                 ::"r"(cluster_addr), "f"(v), "r"(cluster_mbar) : "memory");
 }
 // One request: `sb` adjacent boxes (the map's box is [sb column blocks][128 rows][64 bf16]) starting at weight
 // row `row` and column block `kblock`; they land as sb consecutive swizzled [128][128 B] tiles.
-__device__ __forceinline__ void st_peer_f32(uint32_t local_smem_addr, uint32_t rank, float v)
-{
-    uint32_t ra;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_smem_addr), "r"(rank));
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(v) : "memory");
-}
 __device__ __forceinline__ void tma_load_boxes(uint32_t dst, const CUtensorMap *map, int row, int kblock, uint32_t bar,
                                                unsigned long long policy)
 {
@@ -154,48 +153,61 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-// Dynamic shared memory: this header (5 KB), then a ring of weight boxes [128 rows][128 B], then n_boxes
-// activation boxes [NP rows][128 B]; every box is 1,024-byte aligned.  The partial tile [NP][128] fp32
-// reuses the ring once the products are done (the host checks that it fits).
+// Dynamic shared memory: this header (5 KB), then (small batches) the split-K receive area
+// [8 source ranks][NP / 8 requests][128 features] fp32, then a ring of weight boxes [128 rows][128 B], then
+// n_boxes activation boxes [NP rows][128 B]; every box is 1,024-byte aligned.  For large batches the receive
+// area has no room of its own and reuses the ring once every rank's products are done (the host checks that it fits).
 struct ProjSmemHeader {
     alignas(8) unsigned long long w_full[kProjMaxRing];    // a slot's box has landed
     alignas(8) unsigned long long w_empty[kProjMaxRing];   // the products reading a slot have completed
     alignas(8) unsigned long long mma_done;
+    alignas(8) unsigned long long recv_full;               // every rank's rows of this rank's requests have landed
     uint32_t tmem_base;
     int abort_flag;
     float ssq[kProjMaxBatch];      // stage 0: this rank's sums of squares; stage 1: 1/rms per request
     float part_sum[3][kProjMaxBatch];   // stage 1 prologue
-    float ssq_recv[kProjSplits][kProjMaxBatch];   // stage 0, rank 0: every rank's sums of squares, pushed by their owners
+    float ssq_warp[4][kProjMaxBatch / kProjSplits];   // stage 0: per-warp sums of squares of this rank's requests
     alignas(16) uint16_t gain[kProjMaxBoxes * kProjBoxK];   // stage 1: this K slice of g
 };
 constexpr int kProjHeaderBytes = 5120;
 static_assert(sizeof(ProjSmemHeader) <= kProjHeaderBytes, "header must fit its five kilobytes");
 constexpr int kProjWBoxBytes = kProjTileOut * 128;
-inline size_t proj_smem_bytes(int ring, int n_boxes, int np)
+__host__ __device__ constexpr int proj_recv_bytes(int np) { return kProjSplits * (np / kProjSplits) * kProjTileOut * 4; }
+inline size_t proj_smem_bytes(int ring, int n_boxes, int np, bool own_recv)
 {
-    return 1024 /* alignment slack */ + kProjHeaderBytes + (size_t)ring * kProjWBoxBytes + (size_t)n_boxes * np * 128;
+    return 1024 /* alignment slack */ + kProjHeaderBytes + (own_recv ? proj_recv_bytes(np) : 0) +
+           (size_t)ring * kProjWBoxBytes + (size_t)n_boxes * np * 128;
 }
 // The ring: `slots` requests in flight, each of `sb` adjacent boxes (sb divides the slice's box count).
 // Preferred: the largest request that still leaves room for two CTAs per SM (then every cluster of a product
 // is resident at once), and only then as many slots as fit: the bytes a request reads contiguously per weight
 // row matter more than the ring's depth (one 512-byte-per-row request at a time beat two 256-byte ones in
-// flight).  The ring must also hold the partial tile.  Falls back to one CTA per SM when nothing smaller fits.
-struct ProjRing { int sb, slots; };
-inline ProjRing proj_ring(int n_boxes, int np)
+// flight).  Falls back to one CTA per SM when nothing smaller fits.  The split-K receive area gets room of its
+// own (one cluster barrier fewer) when that costs the ring nothing; otherwise it reuses the ring, which must
+// then be large enough for it.
+struct ProjRing { int sb, slots; bool own_recv; };
+inline ProjRing proj_ring_for(int n_boxes, int np, bool own_recv, size_t budget)
 {
-    const int need = (np * kProjTileOut * 4 + kProjWBoxBytes - 1) / kProjWBoxBytes;   // boxes the partial tile covers
-    for (int pass = 0; pass < 2; ++pass) {
-        const size_t budget = (pass == 0 ? 113 : 227) * 1024;
-        for (int sb = n_boxes; sb >= 1; --sb) {
-            if (n_boxes % sb) continue;
-            const int n_req = n_boxes / sb;
-            for (int slots = (n_req < kProjMaxRing ? n_req : kProjMaxRing); slots >= 1; --slots) {
-                if (sb * slots < need) break;
-                if (proj_smem_bytes(sb * slots, n_boxes, np) <= budget) return ProjRing{sb, slots};
-            }
+    const int need = own_recv ? 0 : (proj_recv_bytes(np) + kProjWBoxBytes - 1) / kProjWBoxBytes;
+    for (int sb = n_boxes; sb >= 1; --sb) {
+        if (n_boxes % sb) continue;
+        const int n_req = n_boxes / sb;
+        for (int slots = (n_req < kProjMaxRing ? n_req : kProjMaxRing); slots >= 1; --slots) {
+            if (sb * slots < need) break;
+            if (proj_smem_bytes(sb * slots, n_boxes, np, own_recv) <= budget) return ProjRing{sb, slots, own_recv};
         }
     }
-    return ProjRing{0, 0};
+    return ProjRing{0, 0, own_recv};
+}
+inline ProjRing proj_ring(int n_boxes, int np)
+{
+    for (int pass = 0; pass < 2; ++pass) {
+        const size_t budget = (pass == 0 ? 113 : 227) * 1024;
+        const ProjRing shared = proj_ring_for(n_boxes, np, false, budget), own = proj_ring_for(n_boxes, np, true, budget);
+        if (own.slots > 0 && own.sb >= shared.sb && own.sb * own.slots >= shared.sb * shared.slots) return own;
+        if (shared.slots > 0) return shared;
+    }
+    return ProjRing{0, 0, false};
 }
 
 template <int STAGE, int NP>
@@ -211,7 +223,10 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
     const int tile = (int)blockIdx.x / kProjSplits;       // which 128 output features
     const int k_slice = A.k_total / kProjSplits, n_boxes = k_slice / kProjBoxK;
     const int sb = A.ring_sb, slots = A.ring_slots, n_req = n_boxes / sb;   // boxes per request, requests in flight, requests
-    uint8_t *w_boxes = smem_al + kProjHeaderBytes;        // [slots][sb][128][128 B]
+    const bool recv_aliased = A.recv_aliased != 0;
+    constexpr int kCols = NP / kProjSplits;               // requests this rank finishes: n = i * 8 + rank, i < kCols
+    uint8_t *w_boxes = smem_al + kProjHeaderBytes + (recv_aliased ? 0 : proj_recv_bytes(NP));   // [slots][sb][128][128 B]
+    float *recv = reinterpret_cast<float *>(recv_aliased ? w_boxes : smem_al + kProjHeaderBytes);   // [8 sources][kCols][128]
     uint8_t *x_boxes = w_boxes + (size_t)slots * sb * kProjWBoxBytes;   // [n_boxes][NP][128 B]
     const int k0 = rank * k_slice;
     volatile int *abort_flag = &sm.abort_flag;
@@ -231,6 +246,8 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
             mbar_init(smem_u32(&sm.w_empty[i]), 1);
         }
         mbar_init(smem_u32(&sm.mma_done), 1);
+        mbar_init(smem_u32(&sm.recv_full), 1);
+        mbar_arrive_expect_tx(smem_u32(&sm.recv_full), (uint32_t)proj_recv_bytes(NP));   // what the eight ranks will send
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         // the first fill of the ring, now: the weight does not depend on anything the stream computed before
@@ -254,12 +271,11 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
         return reinterpret_cast<uint4 *>(x_boxes + (size_t)box * (NP * 128) + m * 128 + ((c ^ (m & 7)) * 16));
     };
     // what the epilogue adds to the product (stage 0), fetched now so that it has long arrived by then
-    const int ep_j = tid & (kProjRowsPerRank - 1), ep_n0 = tid / kProjRowsPerRank;
-    const int ep_o = tile * kProjTileOut + rank * kProjRowsPerRank + ep_j;
-    uint16_t zreg[NP / 8];
+    const int ep_o = tile * kProjTileOut + (tid & (kProjTileOut - 1));   // this thread's output feature
+    uint16_t zreg[kCols];
 #pragma unroll
-    for (int i = 0; i < NP / 8; ++i) {
-        const int n = ep_n0 + 8 * i;
+    for (int i = 0; i < kCols; ++i) {
+        const int n = i * kProjSplits + rank;
         zreg[i] = (STAGE == 0 && is_main && n < A.batch) ? A.z[(size_t)n * A.n_out + ep_o] : (uint16_t)0;
     }
     if (STAGE == 0) {
@@ -358,6 +374,11 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // With a receive area of its own a rank may be written by its peers as soon as it runs and its barriers are
+    // initialised: this arrival, waited for only just before the first remote store, says so.  It orders no data
+    // (relaxed: a releasing arrival cost a microsecond here, and at the top of the kernel so did a relaxed one,
+    // while the cluster's CTAs were still being placed).
+    if (!recv_aliased) cluster_arrive_relaxed();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&sm.tmem_base);
 
     // ---- products: thread 32 issues them box by box as the weight lands, and refills the slots behind them
@@ -401,78 +422,101 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
             mbar_arrive(smem_u32(&sm.mma_done));
         }
     }
-    if (!is_main) {   // helper warps: nothing left to do but keep the cluster barriers' counts whole
-        cluster_sync_all();
-        cluster_sync_all();
+    if (!is_main) {   // helper warps: nothing left to do but keep the cluster barrier's count whole
+        if (recv_aliased) cluster_arrive();
+        cluster_wait();
         return;
     }
     const bool done = mbar_wait(smem_u32(&sm.mma_done), 0, abort_flag) && !*abort_flag;
     if (!done && tid == 0) { sm.abort_flag = 1; atomicOr(A.status, (unsigned)kStatusTimeout); }
     tc_fence_after();
 
-    // ---- this CTA's partial tile: accumulator row t, NP columns -> shared memory [n][128]
-    float *part = reinterpret_cast<float *>(w_boxes);
+    // ---- split-K sum.  Rank r finishes requests n = 8 i + r (all 128 features of each): every rank sends
+    // accumulator row t, column n, straight from tensor memory into recv[its own rank][i][t] of rank n mod 8,
+    // with stores that count their bytes on the receiver's transaction barrier.  The one cluster barrier comes
+    // first: with its own receive area a rank can be written as soon as it runs (it arrived after its staging);
+    // a receive area inside the ring can be written once the rank's products are done.
+    if (recv_aliased) cluster_arrive();
+    cluster_wait();
+    {
+        const uint32_t mine = smem_u32(recv + (size_t)(rank * kCols) * kProjTileOut + tid);
+        const uint32_t bar = smem_u32(&sm.recv_full);
+        uint32_t dst[kProjSplits], dst_bar[kProjSplits];
 #pragma unroll
-    for (int c16 = 0; c16 < NP / 16; ++c16) {
-        float v[16];
-        if (done) {
-            tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c16 * 16), v);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] = 0.f;
+        for (int r = 0; r < kProjSplits; ++r) {
+            dst[r] = peer_addr(mine, (uint32_t)r);
+            dst_bar[r] = peer_addr(bar, (uint32_t)r);
         }
 #pragma unroll
-        for (int i = 0; i < 16; ++i) part[(c16 * 16 + i) * kProjTileOut + tid] = v[i];
+        for (int c16 = 0; c16 < NP / 16; ++c16) {
+            float v[16];
+            if (done) {
+                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c16 * 16), v);
+            } else {      // a rank that gave up still sends (zeros): its peers count on the bytes
+#pragma unroll
+                for (int k = 0; k < 16; ++k) v[k] = 0.f;
+            }
+#pragma unroll
+            for (int k = 0; k < 16; ++k)   // column n = 16 c16 + k: request i = n / 8 of rank n mod 8
+                st_async_f32(dst[k & 7] + (uint32_t)((2 * c16 + (k >> 3)) * kProjTileOut * 4), v[k], dst_bar[k & 7]);
+        }
     }
     tc_fence_before();
-    cluster_sync_all();          // every rank's partial tile is in place
-
-    // ---- sum the eight partials in rank order; this rank finishes output features [16 rank, 16 rank + 16)
+    // Wait for what the eight ranks send here.  The limit is twice any other wait's, and a local abort does not cut
+    // it short: a peer that gives up elsewhere still sends, and this CTA must not leave while stores are on their way.
     {
-        const uint32_t part_addr = smem_u32(part);
-        float pv[NP / 8][kProjSplits];
+        bool landed = false;
+        for (unsigned it = 0; it < 2u * kSpinLimit && !landed; ++it) {
+            landed = mbar_try_wait(smem_u32(&sm.recv_full), 0u);
+            if (!landed && it > 64) __nanosleep(64);
+        }
+        if (!landed && tid == 0) atomicOr(A.status, (unsigned)kStatusTimeout);
+    }
+
+    // ---- the eight partials of this rank's requests, summed in rank order, and the epilogue
+    float sq[kCols];
 #pragma unroll
-        for (int i = 0; i < NP / 8; ++i)        // every remote read is issued before any is summed
+    for (int i = 0; i < kCols; ++i) {
+        const int n = i * kProjSplits + rank;
+        float pv[kProjSplits];
 #pragma unroll
-            for (int c = 0; c < kProjSplits; ++c)
-                pv[i][c] = ld_peer_f32(part_addr + (uint32_t)(((ep_n0 + 8 * i) * kProjTileOut + rank * kProjRowsPerRank + ep_j) * 4),
-                                       (uint32_t)c);
+        for (int c = 0; c < kProjSplits; ++c) pv[c] = recv[(size_t)(c * kCols + i) * kProjTileOut + tid];
+        float y = 0.f;
 #pragma unroll
-        for (int i = 0; i < NP / 8; ++i) {
-            const int n = ep_n0 + 8 * i;
-            float y = 0.f;
-#pragma unroll
-            for (int c = 0; c < kProjSplits; ++c) y += pv[i][c];
-            float sq = 0.f;
-            if (n < A.batch) {
-                if (STAGE == 0) {
-                    const float zf = __uint_as_float((uint32_t)zreg[i] << 16);
-                    const __nv_bfloat16 ub = __float2bfloat16_rn(zf + y);
-                    A.out[(size_t)n * A.n_out + ep_o] = *reinterpret_cast<const uint16_t *>(&ub);
-                    const float uf = __bfloat162float(ub);
-                    sq = uf * uf;
-                } else {
-                    const __nv_bfloat16 qb = __float2bfloat16_rn(y);
-                    A.out[(size_t)n * A.n_out + ep_o] = *reinterpret_cast<const uint16_t *>(&qb);
-                }
-            }
+        for (int c = 0; c < kProjSplits; ++c) y += pv[c];
+        sq[i] = 0.f;
+        if (n < A.batch) {
             if (STAGE == 0) {
-                // sum of squares over the rank's 16 features: the 16 lanes of a half warp, fixed tree
-#pragma unroll
-                for (int off = 8; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
-                if (ep_j == 0) st_peer_f32(smem_u32(&sm.ssq_recv[rank][n]), 0u, sq);   // into rank 0's shared memory
+                const float zf = __uint_as_float((uint32_t)zreg[i] << 16);
+                const __nv_bfloat16 ub = __float2bfloat16_rn(zf + y);
+                A.out[(size_t)n * A.n_out + ep_o] = *reinterpret_cast<const uint16_t *>(&ub);
+                const float uf = __bfloat162float(ub);
+                sq[i] = uf * uf;
+            } else {
+                const __nv_bfloat16 qb = __float2bfloat16_rn(y);
+                A.out[(size_t)n * A.n_out + ep_o] = *reinterpret_cast<const uint16_t *>(&qb);
             }
         }
     }
-    // Partial tiles are no longer read by anybody, and (stage 0) every rank's sums of squares have arrived in
-    // rank 0's shared memory: after this barrier a CTA touches only its own shared memory, so it may leave.
-    cluster_sync_all();
-    if (STAGE == 0 && rank == 0 && tid < NP) {
-        float s = 0.f;
+    if (STAGE == 0) {
+        // sums of squares of the rounded stream over the tile's 128 features, per request: a fixed tree inside
+        // each warp, then the four warps in order
 #pragma unroll
-        for (int c = 0; c < kProjSplits; ++c) s += sm.ssq_recv[c][tid];
-        A.ssq_part[(size_t)tile * kProjMaxBatch + tid] = (tid < A.batch) ? s : 0.f;
+        for (int i = 0; i < kCols; ++i) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) sq[i] += __shfl_xor_sync(0xffffffffu, sq[i], off);
+            if ((tid & 31) == 0) sm.ssq_warp[warp][i] = sq[i];
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kProjThreads) : "memory");   // the 128 main threads (the helpers have left)
+        if (tid < kCols) {
+            const int n = tid * kProjSplits + rank;
+            const float s4 = ((sm.ssq_warp[0][tid] + sm.ssq_warp[1][tid]) + sm.ssq_warp[2][tid]) + sm.ssq_warp[3][tid];
+            A.ssq_part[(size_t)tile * kProjMaxBatch + n] = (n < A.batch) ? s4 : 0.f;
+        }
     }
+    // every warp's reads of tensor memory are complete (they preceded its stores, which have all landed here)
+    asm volatile("bar.sync 1, %0;" ::"n"(kProjThreads) : "memory");
+    tc_fence_after();
     if (warp == 0) tmem_dealloc(tmem, 64);
 }
 
@@ -550,7 +594,8 @@ cudaError_t launch_proj_np(const CUtensorMap &map, const ProjArgs &args, cudaStr
     ProjArgs a2 = args;
     a2.ring_sb = ring.sb;
     a2.ring_slots = ring.slots;
-    const size_t smem = proj_smem_bytes(ring.sb * ring.slots, n_boxes, NP);
+    a2.recv_aliased = ring.own_recv ? 0 : 1;
+    const size_t smem = proj_smem_bytes(ring.sb * ring.slots, n_boxes, NP, ring.own_recv);
     // the attribute is raised once per device to the largest footprint this instantiation can have
     static bool attr_set[64];
     int dev = 0;
