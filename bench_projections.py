@@ -143,9 +143,9 @@ def main():
         "roofline": {"bound": "hbm", "kernel": "proj_kernel (both stages of a pair)", "achieved": achieved,
                      "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "bytes_per_pair": pair_bytes, "traffic": None,
-                     "note": "a pair is two dependent kernels; each spends about 6 us in phases that do not scale with "
-                             "the weight (operand staging, cluster barriers, split-K sum) around a weight stream "
-                             "of 3 us at peak (21 MB at the 4B shape), so the pair is bound by latency, not by HBM"},
+                     "note": "a pair is two dependent kernels; each waits for its weight stream (21 MB at the 4B shape: "
+                             "3 us at peak, 4 to 7 us as a CTA's 64-80 KB requests land) and then spends about 2 us in "
+                             "products, split-K exchange and epilogue, so the pair is bound by latency, not by HBM"},
     }
     if not args.no_cpu_baseline:
         from oracle import qf_oracle as orc

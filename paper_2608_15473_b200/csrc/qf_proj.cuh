@@ -20,16 +20,20 @@
 //     not the whole slice, is resident so that two CTAs fit an SM and every cluster of a product is resident
 //     at once: with the whole slice resident the kernel ran in two waves and took twice as long.
 //   * 256 threads stage the activation slice (the 128 that own accumulator rows plus four helper warps).
-//   * the eight partial tiles are summed over distributed shared memory in rank order (bit-deterministic),
-//     each rank finishing 16 of the tile's 128 output features; two cluster barriers in all.
+//   * split-K sum over distributed shared memory: rank r finishes requests n = 8 i + r.  Every rank sends
+//     accumulator row t, column n, straight from tensor memory into rank (n mod 8)'s receive area with stores
+//     that count their bytes on a transaction barrier of the receiver, which then adds the eight partials in
+//     rank order (bit-deterministic).  One cluster barrier in all, with a relaxed arrival: it only says that
+//     a rank is running (or, for large batches whose receive area reuses the ring, that its products are done).
 //
 // Stage 0 (W_o): X = bf16(a), epilogue u' = bf16(z + Y), plus each tile's sum of squares of the rounded
 // stream per request.  Stage 1 (W_q): X = bf16(g u' / sqrt(mean u'^2 + eps)) built in the prologue from
 // stage 0's outputs, epilogue q = bf16(Y).
 //
 // Every wait on an mbarrier is bounded; a wait that runs out raises the CTA's abort flag and a status bit,
-// the CTA stops computing but still takes part in the cluster barriers, drains its copies and frees its
-// tensor memory.  Every TMA load lands in the shared memory of the CTA that issued it.
+// the CTA stops computing but still takes part in the cluster barrier, sends (zeros) what its peers count on,
+// drains its copies and frees its tensor memory.  Every TMA load lands in the shared memory of the CTA that
+// issued it.
 #pragma once
 
 #include <cuda.h>
@@ -105,7 +109,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
 #pragma unroll
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t cluster_rank()
@@ -423,7 +426,7 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
         }
     }
     if (!is_main) {   // helper warps: nothing left to do but keep the cluster barrier's count whole
-        if (recv_aliased) cluster_arrive();
+        if (recv_aliased) cluster_arrive_relaxed();
         cluster_wait();
         return;
     }
@@ -435,8 +438,9 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
     // accumulator row t, column n, straight from tensor memory into recv[its own rank][i][t] of rank n mod 8,
     // with stores that count their bytes on the receiver's transaction barrier.  The one cluster barrier comes
     // first: with its own receive area a rank can be written as soon as it runs (it arrived after its staging);
-    // a receive area inside the ring can be written once the rank's products are done.
-    if (recv_aliased) cluster_arrive();
+    // a receive area inside the ring can be written once the rank's products are done, which this thread has
+    // seen on mma_done before it arrives (the arrival carries no data, so it need not release anything).
+    if (recv_aliased) cluster_arrive_relaxed();
     cluster_wait();
     {
         const uint32_t mine = smem_u32(recv + (size_t)(rank * kCols) * kProjTileOut + tid);
