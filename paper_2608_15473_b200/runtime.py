@@ -115,3 +115,69 @@ class HostStepper:
         rc = self._fn(*self._args, *self._tail, st)
         if rc != qf.QF_OK:
             raise qf.QFError(rc, "qf_decode_step_host")
+
+
+class CacheSideStack:
+    """The cache side of a stack of layers for one batch of co-resident requests (Section 4): per layer its KV
+    pool, W_o, W_q and the normalisation gain.  A stage of layer l is what the cache side does per token and layer:
+
+        sweep layer l's cache with the query it already holds        (qf_decode_partial)
+        fold in the current token's (k, v), which arrive with z      (qf_combine_self)
+        write them into the cache and advance the lengths            (qf_append_kv)
+        u' = z + W_o a  ->  the wire;  q = W_q N_1(u')  ->  layer l+1 (qf_project_pair)
+
+    Only enqueues library calls (plus one torch add for the lengths); ``capture`` records a whole token, every
+    layer's stage in order, into one CUDA graph whose replays see the lengths grow on the device.
+    """
+
+    def __init__(self, layers, w_o: torch.Tensor, w_q: torch.Tensor, gain: torch.Tensor, eps: float = 1e-6):
+        self.layers = list(layers)
+        L = len(self.layers)
+        d0 = self.layers[0]
+        self.batch, self.n_q = d0.w.batch, d0.w.num_q_heads * d0.w.head_dim
+        self.d_model = int(w_o.shape[1])
+        assert tuple(w_o.shape) == (L, self.d_model, self.n_q) and tuple(w_q.shape) == (L, self.n_q, self.d_model)
+        assert tuple(gain.shape) == (L, self.d_model)
+        for t in (w_o, w_q, gain):
+            assert t.dtype == torch.bfloat16 and t.is_contiguous()
+        self.w_o, self.w_q, self.gain, self.eps = w_o, w_q, gain, float(eps)
+        n = qf.project_workspace_bytes(self.batch, self.d_model, self.n_q)
+        if n == 0:
+            raise qf.QFError(qf.QF_ERR_UNSUPPORTED, "qf_project_workspace_bytes")
+        self.proj_ws = torch.empty(n, dtype=torch.uint8, device=d0.device)
+        self.launches_per_token = 0
+
+    def stage(self, l: int, z, k_new, v_new, u_out, stream=None) -> int:
+        """Enqueue layer l's stage; the next query lands in layer (l + 1) mod L's q buffer.  Returns launches."""
+        dw, nxt = self.layers[l], self.layers[(l + 1) % len(self.layers)]
+        dw.sweep(stream)
+        n = qf.last_launch_count()
+        qf.combine_self(dw.o_part, dw.lse_part, dw.shard_counts, dw.q, k_new, v_new, dw.out, dw.lse, dw.params, stream)
+        qf.append_kv(dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens, k_new, v_new, dw.params, stream)
+        dw.seq_lens.add_(1)
+        qf.project_pair(dw.out.view(self.batch, self.n_q), z, self.w_o[l], self.gain[l], self.w_q[l], u_out,
+                        nxt.q.view(self.batch, self.n_q), self.eps, self.proj_ws, stream)
+        return n + 5
+
+    def token(self, z, k_new, v_new, u_out, stream=None) -> int:
+        """One token through every layer: z, k_new, v_new, u_out are [L, ...] stacks, one slice per layer."""
+        n = 0
+        for l in range(len(self.layers)):
+            n += self.stage(l, z[l], k_new[l], v_new[l], u_out[l], stream)
+        self.launches_per_token = n
+        return n
+
+    def capture(self, z, k_new, v_new, u_out, stream: torch.cuda.Stream) -> torch.cuda.CUDAGraph:
+        """One token as a CUDA graph on ``stream`` (which must be the current stream, so that the length advance
+        is captured too).  Call ``token`` once un-captured before this: the first call of a shape sets kernel
+        attributes and builds descriptors."""
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            self.token(z, k_new, v_new, u_out, stream)
+        return graph
+
+    def status(self) -> int:
+        st = qf.project_status(self.proj_ws)
+        for dw in self.layers:
+            st |= dw.status()
+        return st
