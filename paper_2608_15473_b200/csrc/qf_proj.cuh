@@ -55,7 +55,6 @@ constexpr int kProjBoxK      = 64;    // bf16 per TMA box row: 128 bytes, one sw
 constexpr int kProjMaxBoxes  = 10;    // K / 8 / 64 <= 10, i.e. K <= 5,120
 constexpr int kProjMaxRing   = 4;     // weight requests in flight per CTA, at most
 constexpr int kProjMaxBatch  = 64;
-constexpr int kProjRowsPerRank = kProjTileOut / kProjSplits;   // 16
 
 struct ProjArgs {
     const float *a;            // stage 0: [batch][K] fp32
@@ -221,7 +220,7 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
     uint8_t *smem_al = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     ProjSmemHeader &sm = *reinterpret_cast<ProjSmemHeader *>(smem_al);
     const int tid = threadIdx.x, warp = tid >> 5;
-    const bool is_main = tid < kProjThreads;   // the helper warps leave after the staging (they still join the cluster barriers)
+    const bool is_main = tid < kProjThreads;   // the helper warps leave after the staging (they still join the cluster barrier)
     const int rank = (int)cluster_rank();                 // which eighth of K
     const int tile = (int)blockIdx.x / kProjSplits;       // which 128 output features
     const int k_slice = A.k_total / kProjSplits, n_boxes = k_slice / kProjBoxK;
