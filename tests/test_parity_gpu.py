@@ -245,6 +245,7 @@ def test_long_single_request_many_segments(Hkv, flags):
 def test_small_configs_elementwise():
     for w in (wl.config1(seed=0), wl.config2(seed=1, batch=6), wl.config3(seed=2, batch=4, hi=9000),
               wl.config4(seed=0, ctx=1 << 15, n_shards=16, n_plant=400),
+              wl.config4(seed=1, ctx=1 << 15, n_shards=16, n_plant=400, table="shuffled"),
               wl.config5(seed=0, batch=12, hi=8192)):
         dw = run(w)
         T.compare_all(dw, w, tag=w.name)
