@@ -214,6 +214,25 @@ int qf_combine_self(const float *o_part, const float *lse_part, const int32_t *s
 int qf_append_kv(void *k_cache, void *v_cache, const int32_t *block_table, const int32_t *seq_lens,
                  const void *k_new, const void *v_new,
                  const qf_params *p, void *cuda_stream);
+/*
+ * Section 2, the end of a decode step in ONE launch: qf_combine_self (the
+ * current token folded into the swept shard states: out, lse) and qf_append_kv
+ * (its key and value stored at position seq_lens[b]) together, same arguments,
+ * same results bit for bit.  With advance_lengths != 0 every request whose row
+ * was stored also gets seq_lens[b] += 1, after all of its KV heads have been
+ * placed (a request without a page for the position keeps its length and
+ * stores nothing).  The merge reads neither the cache nor the lengths, so the
+ * two halves share nothing.  All pointers are device pointers; q, k_new,
+ * v_new, k_cache, v_cache 8-byte aligned; shard_counts and block_table may be
+ * NULL.  Errors as qf_combine_self.
+ */
+int qf_fold_append(const float *o_part, const float *lse_part, const int32_t *shard_counts,
+                   const void *q, const void *k_new, const void *v_new,
+                   float *out, float *lse,
+                   void *k_cache, void *v_cache, const int32_t *block_table,
+                   int32_t *seq_lens, int advance_lengths,
+                   const qf_params *p, void *cuda_stream);
+
 
 /*
  * Section 4 ("what each side holds": W_q and W_o live with the cache) and the

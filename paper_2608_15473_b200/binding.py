@@ -39,7 +39,7 @@ EXPORTS = (
     "qf_step_scratch_bytes", "qf_decode_step_host", "qf_read_status", "qf_last_launch_count",
     "qf_set_profile_events", "qf_decode_partial_static", "qf_static_scratch_error",
     "qf_combine_self", "qf_append_kv", "qf_selftest_bounded_wait", "qf_plan_pieces",
-    "qf_project_workspace_bytes", "qf_project_pair", "qf_project_status",
+    "qf_project_workspace_bytes", "qf_project_pair", "qf_project_status", "qf_fold_append",
 )
 
 
@@ -108,6 +108,8 @@ def lib() -> ctypes.CDLL:
         L.qf_decode_partial_static.restype = ctypes.c_int
         L.qf_decode_partial_static.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, vp, vp, pp, vp]
         L.qf_static_scratch_error.restype = ctypes.c_char_p
+        L.qf_fold_append.restype = ctypes.c_int
+        L.qf_fold_append.argtypes = [vp, vp, i32p, vp, vp, vp, vp, vp, vp, vp, i32p, i32p, ctypes.c_int, pp, vp]
         L.qf_project_workspace_bytes.restype = ctypes.c_size_t
         L.qf_project_workspace_bytes.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int]
         L.qf_project_pair.restype = ctypes.c_int
@@ -221,6 +223,17 @@ def append_kv(k_cache, v_cache, block_table, seq_lens, k_new, v_new, p: QFParams
                             _ptr(v_new), ctypes.byref(p), _stream(stream))
     if check and rc != QF_OK:
         raise QFError(rc, "qf_append_kv")
+    return rc
+
+
+def fold_append(o_part, lse_part, shard_counts, q, k_new, v_new, out, lse, k_cache, v_cache, block_table, seq_lens,
+                p: QFParams, advance_lengths: bool = True, stream=None, check: bool = True) -> int:
+    """combine_self and append_kv in one launch; advance_lengths also adds one to the stored requests' lengths."""
+    rc = lib().qf_fold_append(_ptr(o_part), _ptr(lse_part), _ptr(shard_counts), _ptr(q), _ptr(k_new), _ptr(v_new),
+                              _ptr(out), _ptr(lse), _ptr(k_cache), _ptr(v_cache), _ptr(block_table), _ptr(seq_lens),
+                              1 if advance_lengths else 0, ctypes.byref(p), _stream(stream))
+    if check and rc != QF_OK:
+        raise QFError(rc, "qf_fold_append")
     return rc
 
 

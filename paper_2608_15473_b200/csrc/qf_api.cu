@@ -248,6 +248,36 @@ int qf_append_kv(void *k_cache, void *v_cache, const int32_t *block_table, const
     return QF_OK;
 }
 
+int qf_fold_append(const float *o_part, const float *lse_part, const int32_t *shard_counts, const void *q,
+                   const void *k_new, const void *v_new, float *out, float *lse, void *k_cache, void *v_cache,
+                   const int32_t *block_table, int32_t *seq_lens, int advance_lengths, const qf_params *p,
+                   void *cuda_stream)
+{
+    g_last_launches = 0;
+    int rc = validate(p);
+    if (rc != QF_OK) return rc;
+    if (!o_part || !lse_part || !out || !lse || !q || !k_new || !v_new || !k_cache || !v_cache || !seq_lens)
+        return QF_ERR_NULL;
+    if (((uintptr_t)q & 7) || ((uintptr_t)k_new & 7) || ((uintptr_t)v_new & 7) || ((uintptr_t)k_cache & 7) ||
+        ((uintptr_t)v_cache & 7))
+        return QF_ERR_BAD_SHAPE;
+    rc = check_device(nullptr);
+    if (rc != QF_OK) return rc;
+    const qf::DevParams P = dev_params(p);
+    const long long bh = (long long)p->batch * p->num_q_heads;
+    const unsigned fold_blocks = (unsigned)((bh + qf::kCombineWarps - 1) / qf::kCombineWarps);
+    auto kernel = p->max_shards <= 4 ? qf::fold_append_kernel<4> : p->max_shards <= 8 ? qf::fold_append_kernel<8>
+                                                                                      : qf::fold_append_kernel<16>;
+    cudaError_t e = qf::launch_pdl(kernel, dim3(fold_blocks + (unsigned)p->batch), dim3(qf::kCombineWarps * 32), 0,
+                                   (cudaStream_t)cuda_stream, o_part, lse_part, shard_counts, (const uint16_t *)q,
+                                   (const uint16_t *)k_new, (const uint16_t *)v_new, out, lse, (uint16_t *)k_cache,
+                                   (uint16_t *)v_cache, block_table, (int *)seq_lens, advance_lengths != 0 ? 1 : 0,
+                                   fold_blocks, P);
+    if (e != cudaSuccess) return cuda_fail(e, "fold_append_kernel launch");
+    g_last_launches = 1;
+    return QF_OK;
+}
+
 // Carving of the step scratch used by qf_decode_step_host.
 namespace {
 // Device alias of a pinned, mapped host pointer; nullptr for any other kind of memory.

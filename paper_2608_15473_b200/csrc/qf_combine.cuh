@@ -19,17 +19,14 @@ constexpr int kCombineWarps = 4;
 // kCombineBatch: shard vectors in flight per lane (the host picks the smallest that covers max_shards,
 // up to 16: fewer registers, more resident warps when shards are few).
 template <int kCombineBatch>
-__global__ void __launch_bounds__(kCombineWarps * 32)
-combine_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_part,
-               const int *__restrict__ shard_counts, const uint16_t *__restrict__ q,
-               const uint16_t *__restrict__ k_new, const uint16_t *__restrict__ v_new,
-               float *__restrict__ out, float *__restrict__ lse,
-               int batch, int num_q_heads, int num_kv_heads, int max_shards, float sm_scale)
+__device__ __forceinline__ void
+combine_warp(long long bh, const float *__restrict__ o_part, const float *__restrict__ lse_part,
+             const int *__restrict__ shard_counts, const uint16_t *__restrict__ q,
+             const uint16_t *__restrict__ k_new, const uint16_t *__restrict__ v_new,
+             float *__restrict__ out, float *__restrict__ lse,
+             int batch, int num_q_heads, int num_kv_heads, int max_shards, float sm_scale)
 {
-    grid_dependency_wait();
-    grid_launch_dependents();
     const int lane = threadIdx.x & 31;
-    const long long bh = (long long)blockIdx.x * kCombineWarps + (threadIdx.x >> 5);
     if (bh >= (long long)batch * num_q_heads) return;
     const int b = (int)(bh / num_q_heads), h = (int)(bh % num_q_heads);
     // the current token, if any: its score against this head's query and its value row
@@ -123,8 +120,43 @@ combine_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_p
     if (lane == 0) lse[bh] = (M == neg_inf()) ? neg_inf() : M + logf(wsum);
 }
 
+template <int kCombineBatch>
+__global__ void __launch_bounds__(kCombineWarps * 32)
+combine_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_part,
+               const int *__restrict__ shard_counts, const uint16_t *__restrict__ q,
+               const uint16_t *__restrict__ k_new, const uint16_t *__restrict__ v_new,
+               float *__restrict__ out, float *__restrict__ lse,
+               int batch, int num_q_heads, int num_kv_heads, int max_shards, float sm_scale)
+{
+    grid_dependency_wait();
+    grid_launch_dependents();
+    combine_warp<kCombineBatch>((long long)blockIdx.x * kCombineWarps + (threadIdx.x >> 5), o_part, lse_part,
+                                shard_counts, q, k_new, v_new, out, lse, batch, num_q_heads, num_kv_heads, max_shards,
+                                sm_scale);
+}
+
 // The cache write nothing waits on (Section 2): the current token's key and value go to position
 // seq_lens[b] of request b, through the block table.  One warp per (request, KV head).
+// Physical page of position pos of request b, or -1 if the request has no page for it.
+__device__ __forceinline__ long long append_page(const int *__restrict__ block_table, int b, int pos, const DevParams &P)
+{
+    const int lp = pos >> 4;
+    if (pos < 0 || lp >= P.max_pages_per_req) return -1;
+    const long long phys = block_table ? (long long)block_table[(size_t)b * P.max_pages_per_req + lp]
+                                       : (long long)b * P.max_pages_per_req + lp;
+    return (phys < 0 || phys >= P.num_pages) ? -1 : phys;
+}
+// One warp writes the rows of (request b, KV head c) at position pos of physical page phys.
+__device__ __forceinline__ void append_row(uint16_t *__restrict__ k_cache, uint16_t *__restrict__ v_cache,
+                                           const uint16_t *__restrict__ k_new, const uint16_t *__restrict__ v_new,
+                                           int b, int c, int pos, long long phys, const DevParams &P)
+{
+    const int lane = threadIdx.x & 31;
+    const size_t dst = (((size_t)phys * P.num_kv_heads + c) * kPageSize + (pos & 15)) * kHeadDim + lane * 4;
+    const size_t src = ((size_t)b * P.num_kv_heads + c) * kHeadDim + lane * 4;
+    *reinterpret_cast<uint2 *>(k_cache + dst) = *reinterpret_cast<const uint2 *>(k_new + src);
+    *reinterpret_cast<uint2 *>(v_cache + dst) = *reinterpret_cast<const uint2 *>(v_new + src);
+}
 __global__ void __launch_bounds__(kCombineWarps * 32)
 append_kv_kernel(uint16_t *__restrict__ k_cache, uint16_t *__restrict__ v_cache,
                  const int *__restrict__ block_table, const int *__restrict__ seq_lens,
@@ -132,20 +164,44 @@ append_kv_kernel(uint16_t *__restrict__ k_cache, uint16_t *__restrict__ v_cache,
 {
     grid_dependency_wait();
     grid_launch_dependents();
-    const int lane = threadIdx.x & 31;
     const long long bc = (long long)blockIdx.x * kCombineWarps + (threadIdx.x >> 5);
     if (bc >= (long long)P.batch * P.num_kv_heads) return;
     const int b = (int)(bc / P.num_kv_heads), c = (int)(bc % P.num_kv_heads);
     const int pos = seq_lens[b];
-    const int lp = pos >> 4;
-    if (pos < 0 || lp >= P.max_pages_per_req) return;   // no page for this position: nothing is written
-    const long long phys = block_table ? (long long)block_table[(size_t)b * P.max_pages_per_req + lp]
-                                       : (long long)b * P.max_pages_per_req + lp;
-    if (phys < 0 || phys >= P.num_pages) return;         // unallocated page: nothing is written
-    const size_t dst = (((size_t)phys * P.num_kv_heads + c) * kPageSize + (pos & 15)) * kHeadDim + lane * 4;
-    const size_t src = (size_t)bc * kHeadDim + lane * 4;
-    *reinterpret_cast<uint2 *>(k_cache + dst) = *reinterpret_cast<const uint2 *>(k_new + src);
-    *reinterpret_cast<uint2 *>(v_cache + dst) = *reinterpret_cast<const uint2 *>(v_new + src);
+    const long long phys = append_page(block_table, b, pos, P);
+    if (phys < 0) return;   // no page for this position, or an unallocated one: nothing is written
+    append_row(k_cache, v_cache, k_new, v_new, b, c, pos, phys, P);
+}
+
+// The end of a decode step in one launch (Section 2): the first fold_blocks CTAs fold the current token into the
+// swept shard states (the merge above), the others, one per request, write the token's key and value into the cache
+// at position seq_lens[b] and, if asked, advance that length — after every row of the request has been placed, and
+// only if the position had a page.  The merge reads neither the cache nor the lengths, so the two halves share nothing.
+template <int kCombineBatch>
+__global__ void __launch_bounds__(kCombineWarps * 32)
+fold_append_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_part,
+                   const int *__restrict__ shard_counts, const uint16_t *__restrict__ q,
+                   const uint16_t *__restrict__ k_new, const uint16_t *__restrict__ v_new,
+                   float *__restrict__ out, float *__restrict__ lse, uint16_t *__restrict__ k_cache,
+                   uint16_t *__restrict__ v_cache, const int *__restrict__ block_table, int *__restrict__ seq_lens,
+                   int advance, unsigned fold_blocks, DevParams P)
+{
+    grid_dependency_wait();
+    grid_launch_dependents();
+    if (blockIdx.x < fold_blocks) {
+        combine_warp<kCombineBatch>((long long)blockIdx.x * kCombineWarps + (threadIdx.x >> 5), o_part, lse_part,
+                                    shard_counts, q, k_new, v_new, out, lse, P.batch, P.num_q_heads, P.num_kv_heads,
+                                    P.max_shards, P.sm_scale);
+        return;
+    }
+    const int b = (int)(blockIdx.x - fold_blocks);
+    const int pos = seq_lens[b];
+    const long long phys = append_page(block_table, b, pos, P);
+    if (phys < 0) return;                       // the same for every thread of the CTA
+    for (int c = threadIdx.x >> 5; c < P.num_kv_heads; c += kCombineWarps)
+        append_row(k_cache, v_cache, k_new, v_new, b, c, pos, phys, P);
+    __syncthreads();                            // every warp has read the length and placed its rows
+    if (advance && threadIdx.x == 0) seq_lens[b] = pos + 1;
 }
 
 // Staging of a decode step's inputs from pinned, mapped host memory: the kernel reads the host buffers

@@ -122,12 +122,12 @@ class CacheSideStack:
     pool, W_o, W_q and the normalisation gain.  A stage of layer l is what the cache side does per token and layer:
 
         sweep layer l's cache with the query it already holds        (qf_decode_partial)
-        fold in the current token's (k, v), which arrive with z      (qf_combine_self)
-        write them into the cache and advance the lengths            (qf_append_kv)
+        fold in the current token's (k, v), which arrive with z,
+        write them into the cache and advance the lengths            (qf_fold_append)
         u' = z + W_o a  ->  the wire;  q = W_q N_1(u')  ->  layer l+1 (qf_project_pair)
 
-    Only enqueues library calls (plus one torch add for the lengths); ``capture`` records a whole token, every
-    layer's stage in order, into one CUDA graph whose replays see the lengths grow on the device.
+    Only enqueues library calls; ``capture`` records a whole token, every layer's stage in order, into one CUDA
+    graph whose replays see the lengths grow on the device.
     """
 
     def __init__(self, layers, w_o: torch.Tensor, w_q: torch.Tensor, gain: torch.Tensor, eps: float = 1e-6):
@@ -152,12 +152,11 @@ class CacheSideStack:
         dw, nxt = self.layers[l], self.layers[(l + 1) % len(self.layers)]
         dw.sweep(stream)
         n = qf.last_launch_count()
-        qf.combine_self(dw.o_part, dw.lse_part, dw.shard_counts, dw.q, k_new, v_new, dw.out, dw.lse, dw.params, stream)
-        qf.append_kv(dw.k_cache, dw.v_cache, dw.block_table, dw.seq_lens, k_new, v_new, dw.params, stream)
-        dw.seq_lens.add_(1)
+        qf.fold_append(dw.o_part, dw.lse_part, dw.shard_counts, dw.q, k_new, v_new, dw.out, dw.lse, dw.k_cache,
+                       dw.v_cache, dw.block_table, dw.seq_lens, dw.params, advance_lengths=True, stream=stream)
         qf.project_pair(dw.out.view(self.batch, self.n_q), z, self.w_o[l], self.gain[l], self.w_q[l], u_out,
                         nxt.q.view(self.batch, self.n_q), self.eps, self.proj_ws, stream)
-        return n + 5
+        return n + 3
 
     def token(self, z, k_new, v_new, u_out, stream=None) -> int:
         """One token through every layer: z, k_new, v_new, u_out are [L, ...] stacks, one slice per layer."""
@@ -168,9 +167,8 @@ class CacheSideStack:
         return n
 
     def capture(self, z, k_new, v_new, u_out, stream: torch.cuda.Stream) -> torch.cuda.CUDAGraph:
-        """One token as a CUDA graph on ``stream`` (which must be the current stream, so that the length advance
-        is captured too).  Call ``token`` once un-captured before this: the first call of a shape sets kernel
-        attributes and builds descriptors."""
+        """One token as a CUDA graph on ``stream``.  Call ``token`` once un-captured before this: the first call
+        of a shape sets kernel attributes and builds descriptors."""
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=stream):
             self.token(z, k_new, v_new, u_out, stream)

@@ -133,6 +133,39 @@ def test_append_skips_requests_without_a_page():
     assert int(diff.sum()) == int(diff[p1, :, 5].sum()) and int(diff[p1, :, 5].sum()) > 0
 
 
+@pytest.mark.parametrize("advance", [True, False])
+def test_fold_append_in_one_launch_equals_the_two_calls(advance):
+    # request 1 is full (its next position needs a page its table row does not have): nothing stored, length kept
+    lens = [0, 16, 15, 16, 17, 700, 2500]
+    cap = [16, 16, 15, 32, 17, 700, 2500]       # tokens each request has pages for
+    w = wl.make_workload("fa", cap, [wl.fixed_shards(c, 600) for c in cap], 32, 8, seed=89, max_pages_per_req=200)
+    w.seq_lens = np.asarray(lens, np.int32)
+    k_new, v_new = new_token(w, 13)
+    dk, dv = dev_bf16(k_new), dev_bf16(v_new)
+    a, f = DeviceWorkload(w), DeviceWorkload(w)
+    for dw in (a, f):
+        dw.seq_lens.copy_(torch.from_numpy(w.seq_lens).cuda())
+        dw.sweep()
+    qf.combine_self(a.o_part, a.lse_part, a.shard_counts, a.q, dk, dv, a.out, a.lse, a.params)
+    qf.append_kv(a.k_cache, a.v_cache, a.block_table, a.seq_lens, dk, dv, a.params)
+    qf.fold_append(f.o_part, f.lse_part, f.shard_counts, f.q, dk, dv, f.out, f.lse, f.k_cache, f.v_cache,
+                   f.block_table, f.seq_lens, f.params, advance_lengths=advance)
+    assert qf.last_launch_count() == 1
+    torch.cuda.synchronize()
+    for x, y in ((a.out, f.out), (a.lse, f.lse)):
+        assert torch.equal(x.view(torch.int32), y.view(torch.int32))
+    for x, y in ((a.k_cache, f.k_cache), (a.v_cache, f.v_cache)):
+        assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+    stored = np.array([L // 16 < (c + 15) // 16 for L, c in zip(lens, cap)])
+    assert stored.tolist() == [True, False, True, True, True, True, True]
+    want = np.asarray(lens) + (stored if advance else 0)
+    assert np.array_equal(f.seq_lens.cpu().numpy(), want)
+    # and the stored rows are the token's, where they belong
+    kc = f.k_cache.view(torch.int16).cpu().numpy().view(np.uint16)
+    for b in np.nonzero(stored)[0]:
+        assert np.array_equal(kc[w.block_table[b, lens[b] // 16], :, lens[b] % 16], k_new[b])
+
+
 def test_decode_loop_is_a_fold_over_steps():
     # Twenty decode steps: sweep the cache, fold the current token in, append it, advance.  After every step
     # the result must equal attention over all positions so far plus the current one (the appendix's fold).
