@@ -115,15 +115,19 @@ def sweep_kernel_bytes(w) -> int:
             w.batch * w.num_q_heads * D * 2 + n_sh * w.num_q_heads * (D + 2) * 4)
 
 
-def oracle_pass(w, orc, sample_requests=None):
-    """The CPU oracle over (a sample of) the workload: shard states, then the merge."""
+def oracle_pass(w, orc, sample_requests=None, results=None):
+    """The CPU oracle over (a sample of) the workload: shard states, then the merge.  `results`, a list, receives
+    the merged (out, lse) of a whole-workload pass."""
     sh = orc.Shape(batch=w.batch, num_q_heads=w.num_q_heads, num_kv_heads=w.num_kv_heads,
                    max_pages_per_req=w.max_pages_per_req, max_shards=w.max_shards)
     if sample_requests is None:
         t0 = time.perf_counter()
         op, mp, lp = orc.decode_partial(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.shard_ranges, sh)
-        orc.combine(op, lp, w.shard_counts, sh)
-        return time.perf_counter() - t0, w.algorithmic_bytes(), w.swept_tokens()
+        merged = orc.combine(op, lp, w.shard_counts, sh)
+        dt = time.perf_counter() - t0
+        if results is not None:
+            results.extend(merged[:2])
+        return dt, w.algorithmic_bytes(), w.swept_tokens()
     # bounded sample: the first n requests (all their shards and heads)
     n = sample_requests
     sh.batch = n
@@ -302,7 +306,18 @@ def run_cuda(args):
         if not args.no_cpu_baseline and not args.profile_mode and world == 1:
             from oracle import qf_oracle as orc
             orc.build()
-            dt, nb, ntok = oracle_pass(w, orc)
+            merged = []
+            dt, nb, ntok = oracle_pass(w, orc, results=merged)
+            # the oracle's pass is here anyway: what the timed configuration computed, against it
+            ref_out, ref_lse = merged
+            got_out, got_lse = dw.out.cpu().numpy().astype(np.float64), dw.lse.cpu().numpy().astype(np.float64)
+            fin = np.isfinite(ref_lse)
+            line["parity"] = {"max_abs_out": float(np.abs(got_out - ref_out).max()),
+                              "max_rel_lse": float((np.abs(got_lse[fin] - ref_lse[fin]) /
+                                                    np.maximum(1.0, np.abs(ref_lse[fin]))).max()) if fin.any() else 0.0,
+                              "inf_pattern_matches": bool(np.array_equal(np.isfinite(got_lse), fin)),
+                              "tolerance": {"out_max_abs": 2e-3, "lse_rel": 1e-5},
+                              "against": "the CPU oracle's merged result over the whole workload (every request and head)"}
             line["cpu_baseline"] = {"value": nb / dt / 1e9, "unit": "GB/s", "cores": orc.num_threads(),
                                     "kind": "oracle", "seconds": dt,
                                     "sample": f"the whole workload once: {w.batch} requests, {ntok} cached tokens, "
