@@ -203,7 +203,7 @@ def run_cuda(args):
 
     # every rank owns its own batch of requests (weak scaling): seed + rank
     w = wl.CONFIGS[args.workload](seed=args.seed + rank)
-    dw = DeviceWorkload(w, device=device)
+    dw = DeviceWorkload(w, device=device, flags=qf.QF_FLAG_KV_NHD if args.kv_layout == "nhd" else 0)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -284,7 +284,8 @@ def run_cuda(args):
             "config": {"workload": workload_name(args.workload), "seed": args.seed, "requests_per_gpu": w.batch,
                        "cached_tokens_per_gpu": w.total_tokens, "num_pages": w.num_pages,
                        "l2": "inputs larger than L2 (KV bytes per step >> 126 MB), no flush needed",
-                       "parallelism": f"requests sharded over {world} GPU(s), no collective"},
+                       "parallelism": f"requests sharded over {world} GPU(s), no collective",
+                       "kv_layout": "[page, Hkv, 16, D]" if args.kv_layout == "hnd" else "[page, 16, Hkv, D]"},
             "clocks": clocks.summary(),
             "e2e": {"value": whole_job_throughput(tot_bytes, e2e_ms / args.steps), "unit": "GB/s",
                     "h2d_bytes_per_step": hs.h2d_bytes, "d2h_bytes_per_step": hs.d2h_bytes,
@@ -336,6 +337,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--kv-layout", default="hnd", choices=["hnd", "nhd"],
+                    help="page layout of the KV pools: head-major (default, the headline) or token-major")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile-mode", action="store_true",
                     help="for runs under a profiler: no padding loop, one end-to-end step, no CPU baseline")

@@ -37,7 +37,12 @@
  *   q            bf16  [B, Hq, D]
  *   k_cache,
  *   v_cache      bf16  [num_pages, Hkv, page_size, D]   (one (page, KV head)
- *                       block is page_size*D contiguous elements)
+ *                       block is page_size*D contiguous elements), or, with
+ *                       QF_FLAG_KV_NHD, token-major pages
+ *                       [num_pages, page_size, Hkv, D] (the rows of one KV
+ *                       head of a page are Hkv*D elements apart).  The paper
+ *                       says only "paged"; both are layouts serving stacks
+ *                       keep, and the results are the same bit for bit.
  *   block_table  int32 [B, max_pages_per_req]  logical page -> physical page.
  *                       May be NULL: then request b's logical page p is
  *                       physical page b*max_pages_per_req + p.
@@ -100,11 +105,15 @@ enum {
 enum {
     QF_FLAG_CHECK_BOUNDS  = 1, /* range-check page indices on the device           */
     QF_FLAG_SIMPLE_KERNEL = 2, /* use the plain-load sweep kernel (validation aid) */
-    QF_FLAG_DRAW_ALWAYS   = 8  /* default sweep kernel only: hand out the tail of the work
+    QF_FLAG_DRAW_ALWAYS   = 8, /* default sweep kernel only: hand out the tail of the work
                                   as drawn chunks however short the sweep is (by default
                                   only sweeps long enough to gain from it do).  Same
                                   results up to fp32 summation order; lets small tests
                                   reach the drawn-chunk path                             */
+    QF_FLAG_KV_NHD        = 16 /* k_cache and v_cache are [num_pages, page_size, Hkv, D]
+                                  (token-major pages) instead of [num_pages, Hkv,
+                                  page_size, D]; honoured by every call that touches
+                                  the cache (sweep, cache write, host step)            */
 };
 
 /* qf_read_status bits */

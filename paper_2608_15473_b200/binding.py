@@ -29,6 +29,7 @@ QF_STATIC_SCRATCH_BYTES = 8 << 20
 QF_FLAG_CHECK_BOUNDS = 1
 QF_FLAG_SIMPLE_KERNEL = 2
 QF_FLAG_DRAW_ALWAYS = 8
+QF_FLAG_KV_NHD = 16
 
 QF_STATUS_BAD_PAGE = 1
 QF_STATUS_TIMEOUT = 2

@@ -59,6 +59,7 @@ qf::DevParams dev_params(const qf_params *p)
     d.out_shard0 = p->out_shards > 0 ? p->out_shard_offset : 0;
     d.check_bounds = (p->flags & QF_FLAG_CHECK_BOUNDS) ? 1 : 0;
     d.draw_always = (p->flags & QF_FLAG_DRAW_ALWAYS) ? 1 : 0;
+    d.kv_nhd = (p->flags & QF_FLAG_KV_NHD) ? 1 : 0;
     d.num_pages = p->num_pages;
     d.sm_scale = p->sm_scale > 0.f ? p->sm_scale : 1.0f / std::sqrt((float)p->head_dim);
     return d;

@@ -152,7 +152,7 @@ __device__ __forceinline__ void append_row(uint16_t *__restrict__ k_cache, uint1
                                            int b, int c, int pos, long long phys, const DevParams &P)
 {
     const int lane = threadIdx.x & 31;
-    const size_t dst = (((size_t)phys * P.num_kv_heads + c) * kPageSize + (pos & 15)) * kHeadDim + lane * 4;
+    const size_t dst = kv_row_offset(P, phys, c, pos & 15) + lane * 4;
     const size_t src = ((size_t)b * P.num_kv_heads + c) * kHeadDim + lane * 4;
     *reinterpret_cast<uint2 *>(k_cache + dst) = *reinterpret_cast<const uint2 *>(k_new + src);
     *reinterpret_cast<uint2 *>(v_cache + dst) = *reinterpret_cast<const uint2 *>(v_new + src);

@@ -27,9 +27,17 @@ struct DevParams {
     int out_shard0;          // output slot of this call's shard 0
     int check_bounds;
     int draw_always;         // cut the tail into drawn chunks however short the sweep is
+    int kv_nhd;              // pools are token-major [page][16][Hkv][D] instead of head-major [page][Hkv][16][D]
     long long num_pages;
     float sm_scale;
 };
+
+// Element offset of the row of (physical page, KV head c, slot t of the page) in a KV pool.
+__host__ __device__ __forceinline__ size_t kv_row_offset(const DevParams &P, long long phys, int c, int t)
+{
+    return P.kv_nhd ? (((size_t)phys * kPageSize + t) * P.num_kv_heads + c) * kHeadDim
+                    : (((size_t)phys * P.num_kv_heads + c) * kPageSize + t) * kHeadDim;
+}
 
 // Programmatic dependent launch: every kernel of the path is launched with the programmatic-stream-
 // serialization attribute, so its CTAs may become resident while the previous kernel of the stream is

@@ -67,6 +67,16 @@ __device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap *m
         " [%0], [%1, {%2, %3, %4}], [%5], %6;"
         ::"r"(dst), "l"(map), "r"(0), "r"(row), "r"(0), "r"(bar), "l"(policy) : "memory");
 }
+// The same box from a token-major pool: 16 rows of one KV head, Hkv rows apart (a 4-D view: channel half,
+// KV head, token, half of the row).
+__device__ __forceinline__ void tma_load_page_nhd(uint32_t dst, const CUtensorMap *map, int kv_head, int token_row,
+                                                  uint32_t bar, unsigned long long policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+        ::"r"(dst), "l"(map), "r"(0), "r"(kv_head), "r"(token_row), "r"(0), "r"(bar), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
 {
     asm volatile(

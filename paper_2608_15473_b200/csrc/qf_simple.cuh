@@ -51,7 +51,7 @@ sweep_simple_kernel(const uint16_t *__restrict__ q, const uint16_t *__restrict__
             if (lane == 0) epoch_or(header + kHdrStatus, epoch, kStatusBadPage);
             continue;
         }
-        const size_t row = (((size_t)phys * Hkv + c) * kPageSize + slot) * kHeadDim + lane * 4;
+        const size_t row = kv_row_offset(P, phys, c, slot) + lane * 4;
         const uint2 kw = *reinterpret_cast<const uint2 *>(k_cache + row);
         const uint2 vw = *reinterpret_cast<const uint2 *>(v_cache + row);
         const float k0 = bf16lo_to_f32(kw.x), k1 = bf16hi_to_f32(kw.x);

@@ -449,8 +449,11 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                     }
                     __syncwarp();
                     if (issuer) {
-                        const int row = (phys * Hkv + c) * kPageSize;
-                        tma_load_page(smem_u32(&sm.kv[stage][part][i][0]), part ? &v_map : &k_map, row, full, kv_policy);
+                        const uint32_t dst = smem_u32(&sm.kv[stage][part][i][0]);
+                        if (P.kv_nhd)
+                            tma_load_page_nhd(dst, part ? &v_map : &k_map, c, phys * kPageSize, full, kv_policy);
+                        else
+                            tma_load_page(dst, part ? &v_map : &k_map, (phys * Hkv + c) * kPageSize, full, kv_policy);
                     }
                     if (first && lane == 0)
                         bulk_load_1d(smem_u32(&sm.q[stage][0]), q + ((size_t)b * Hq + (size_t)c * G) * kHeadDim,
@@ -661,23 +664,26 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapFloatOOBfill);
 
 // A [2 halves, rows, 64] bf16 view of a KV pool, one 4 KB box per (page, KV head), 128B swizzle.
-// box_rows = 16 boxes one (page, KV head) block (4 KB); 128 boxes eight heads of a page (32 KB).
+// box_rows = 16 boxes one (page, KV head) block (4 KB).  For a token-major pool (nhd) the view has a fourth
+// dimension, the KV head between the channel half and the token row, and a box takes 16 token rows of one head,
+// Hkv rows apart; either way the box lands in shared memory as [half][row][128 B].
 inline int make_pool_map(CUtensorMap *out, const void *pool, long long num_pages, int num_kv_heads, int box_rows,
-                         char *msg, size_t msg_len)
+                         bool nhd, char *msg, size_t msg_len)
 {
     static EncodeTiledFn encode = nullptr;
     static std::mutex mu;
-    struct Entry { const void *pool; long long pages; int heads; int rows; CUtensorMap map; };
+    struct Entry { const void *pool; long long pages; int heads; int rows; CUtensorMap map; };   // rows < 0: token-major
     // One descriptor per (pointer, shape), hashed by the pointer: a decode loop walks every layer's pools each
     // step, so the cache holds a whole model's worth and a lookup is a handful of probes, not a scan.
     constexpr int kCacheEntries = 1024, kProbes = 8;
     static Entry cache[kCacheEntries];   // zero-initialised: pool == nullptr marks a free entry
     const size_t home = (size_t)(((uintptr_t)pool >> 8) * 0x9E3779B97F4A7C15ull >> 40) % kCacheEntries;
     std::lock_guard<std::mutex> lock(mu);
+    const int key_rows = nhd ? -box_rows : box_rows;
     size_t victim = home;
     for (int i = 0; i < kProbes; ++i) {
         Entry &c = cache[(home + i) % kCacheEntries];
-        if (c.pool == pool && c.pages == num_pages && c.heads == num_kv_heads && c.rows == box_rows) {
+        if (c.pool == pool && c.pages == num_pages && c.heads == num_kv_heads && c.rows == key_rows) {
             *out = c.map;
             return 0;
         }
@@ -698,9 +704,14 @@ inline int make_pool_map(CUtensorMap *out, const void *pool, long long num_pages
     const cuuint64_t dims[3] = {64, (cuuint64_t)num_pages * num_kv_heads * kPageSize, 2};
     const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, 128};
     const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 2};
-    const cuuint32_t estr[3] = {1, 1, 1};
+    // token-major: channels, KV heads (256 B apart), token rows (Hkv x 256 B apart), halves (128 B apart)
+    const cuuint64_t dims4[4] = {64, (cuuint64_t)num_kv_heads, (cuuint64_t)num_pages * kPageSize, 2};
+    const cuuint64_t strides4[3] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)num_kv_heads * kHeadDim * 2, 128};
+    const cuuint32_t box4[4] = {64, 1, (cuuint32_t)box_rows, 2};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
     CUtensorMap map;
-    CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(pool), dims, strides, box,
+    CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, nhd ? 4 : 3, const_cast<void *>(pool),
+                        nhd ? dims4 : dims, nhd ? strides4 : strides, nhd ? box4 : box,
                         estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -708,7 +719,7 @@ inline int make_pool_map(CUtensorMap *out, const void *pool, long long num_pages
         return -1;
     }
     Entry &slot = cache[victim];   // a free entry among the probes, else the home entry is replaced
-    slot.pool = pool; slot.pages = num_pages; slot.heads = num_kv_heads; slot.rows = box_rows; slot.map = map;
+    slot.pool = pool; slot.pages = num_pages; slot.heads = num_kv_heads; slot.rows = key_rows; slot.map = map;
     *out = map;
     return 0;
 }
@@ -774,8 +785,8 @@ inline int launch_sweep(const void *q, const void *k_cache, const void *v_cache,
                         cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1, char *msg, size_t msg_len, int *launches)
 {
     CUtensorMap kmap, vmap;
-    if (make_pool_map(&kmap, k_cache, P.num_pages, P.num_kv_heads, kPageSize, msg, msg_len)) return -5;
-    if (make_pool_map(&vmap, v_cache, P.num_pages, P.num_kv_heads, kPageSize, msg, msg_len)) return -5;
+    if (make_pool_map(&kmap, k_cache, P.num_pages, P.num_kv_heads, kPageSize, P.kv_nhd != 0, msg, msg_len)) return -5;
+    if (make_pool_map(&vmap, v_cache, P.num_pages, P.num_kv_heads, kPageSize, P.kv_nhd != 0, msg, msg_len)) return -5;
     const int n_ctas = sm_count < kMaxSweepCtas ? sm_count : kMaxSweepCtas;
     switch (P.group) {
     case 1: return launch_sweep_g<1>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);

@@ -33,8 +33,12 @@ class DeviceWorkload:
         B, Hq, D, S = w.batch, w.num_q_heads, w.head_dim, w.max_shards
         self.params = qf.params(B, Hq, w.num_kv_heads, w.max_pages_per_req, S, w.num_pages, flags=flags)
         self.q = _to_dev(w.q.view(np.int16), dev, torch.bfloat16)
-        self.k_cache = _to_dev(w.k_cache.view(np.int16), dev, torch.bfloat16)
-        self.v_cache = _to_dev(w.v_cache.view(np.int16), dev, torch.bfloat16)
+        # the host workload keeps pages head-major [page, Hkv, 16, D]; with QF_FLAG_KV_NHD the device copy is
+        # the token-major [page, 16, Hkv, D] arrangement of the same values
+        self.kv_nhd = bool(flags & qf.QF_FLAG_KV_NHD)
+        order = (0, 2, 1, 3) if self.kv_nhd else (0, 1, 2, 3)
+        self.k_cache = _to_dev(w.k_cache.view(np.int16).transpose(order), dev, torch.bfloat16)
+        self.v_cache = _to_dev(w.v_cache.view(np.int16).transpose(order), dev, torch.bfloat16)
         self.block_table = None if identity_table_as_null else _to_dev(w.block_table, dev)
         self.seq_lens = _to_dev(w.seq_lens, dev)
         self.shard_ranges = _to_dev(w.shard_ranges, dev)
@@ -49,6 +53,12 @@ class DeviceWorkload:
             raise qf.QFError(qf.QF_ERR_UNSUPPORTED, "qf_workspace_bytes")
         self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
         assert self.workspace.data_ptr() % 256 == 0
+
+    def cache_head_major(self, which: str = "k") -> np.ndarray:
+        """Host copy (uint16 bit patterns) of a device pool in the host workload's [page, Hkv, 16, D] order."""
+        t = self.k_cache if which == "k" else self.v_cache
+        a = t.view(torch.int16).cpu().numpy().view(np.uint16)
+        return np.ascontiguousarray(a.transpose(0, 2, 1, 3)) if self.kv_nhd else a
 
     def poison_outputs(self) -> None:
         for t in (self.o_part, self.m_part, self.lse_part, self.out, self.lse):

@@ -33,7 +33,11 @@ def run(w, flags=0, null_table=False):
 # "draw": the unit kernel with its drawn-chunk tail forced on (by default only long sweeps use it)
 KERNELS = [pytest.param((0, 16), id="unit16"), pytest.param((0, 8), id="unit8"),
            pytest.param((0, 2), id="unit2"), pytest.param((qf.QF_FLAG_SIMPLE_KERNEL, 2), id="simple"),
-           pytest.param((qf.QF_FLAG_DRAW_ALWAYS, 8), id="draw8"), pytest.param((qf.QF_FLAG_DRAW_ALWAYS, 2), id="draw2")]
+           pytest.param((qf.QF_FLAG_DRAW_ALWAYS, 8), id="draw8"), pytest.param((qf.QF_FLAG_DRAW_ALWAYS, 2), id="draw2"),
+           # token-major pages (the device copy is rearranged by DeviceWorkload; the oracle sees the same values)
+           pytest.param((qf.QF_FLAG_KV_NHD, 8), id="nhd8"), pytest.param((qf.QF_FLAG_KV_NHD, 2), id="nhd2"),
+           pytest.param((qf.QF_FLAG_KV_NHD | qf.QF_FLAG_SIMPLE_KERNEL, 2), id="simple-nhd"),
+           pytest.param((qf.QF_FLAG_KV_NHD | qf.QF_FLAG_DRAW_ALWAYS, 8), id="draw8-nhd")]
 
 
 # T1: every short length, both group sizes, shuffled table: tail-page masking, first-tile guard
@@ -371,10 +375,11 @@ def test_host_step_matches_device_path(pinned):
 
 
 # T8: the benchmark configurations at full size, sampled outputs
-@pytest.mark.parametrize("cfg,seed", [(2, 0), (3, 0), (4, 0), (5, 0), (2, 1), (2, 2), (3, 1), (3, 2), (4, 1)])
-def test_full_size_configs_sampled(cfg, seed):
+@pytest.mark.parametrize("cfg,seed,flags", [(2, 0, 0), (3, 0, 0), (4, 0, 0), (5, 0, 0), (2, 1, 0), (2, 2, 0), (3, 1, 0),
+                                            (3, 2, 0), (4, 1, 0), (3, 0, qf.QF_FLAG_KV_NHD), (2, 0, qf.QF_FLAG_KV_NHD)])
+def test_full_size_configs_sampled(cfg, seed, flags):
     w = wl.CONFIGS[cfg](seed=seed)
-    dw = run(w)
+    dw = run(w, flags)
     errs = T.compare_sampled(dw, w, seed=cfg + 10 * seed, tag=w.name)
     print(w.name, errs)
     assert dw.status() == 0

@@ -133,8 +133,9 @@ def test_append_skips_requests_without_a_page():
     assert int(diff.sum()) == int(diff[p1, :, 5].sum()) and int(diff[p1, :, 5].sum()) > 0
 
 
+@pytest.mark.parametrize("layout", [0, qf.QF_FLAG_KV_NHD])
 @pytest.mark.parametrize("advance", [True, False])
-def test_fold_append_in_one_launch_equals_the_two_calls(advance):
+def test_fold_append_in_one_launch_equals_the_two_calls(advance, layout):
     # request 1 is full (its next position needs a page its table row does not have): nothing stored, length kept
     lens = [0, 16, 15, 16, 17, 700, 2500]
     cap = [16, 16, 15, 32, 17, 700, 2500]       # tokens each request has pages for
@@ -142,7 +143,7 @@ def test_fold_append_in_one_launch_equals_the_two_calls(advance):
     w.seq_lens = np.asarray(lens, np.int32)
     k_new, v_new = new_token(w, 13)
     dk, dv = dev_bf16(k_new), dev_bf16(v_new)
-    a, f = DeviceWorkload(w), DeviceWorkload(w)
+    a, f = DeviceWorkload(w, flags=layout), DeviceWorkload(w, flags=layout)
     for dw in (a, f):
         dw.seq_lens.copy_(torch.from_numpy(w.seq_lens).cuda())
         dw.sweep()
@@ -161,12 +162,13 @@ def test_fold_append_in_one_launch_equals_the_two_calls(advance):
     want = np.asarray(lens) + (stored if advance else 0)
     assert np.array_equal(f.seq_lens.cpu().numpy(), want)
     # and the stored rows are the token's, where they belong
-    kc = f.k_cache.view(torch.int16).cpu().numpy().view(np.uint16)
+    kc = f.cache_head_major("k")
     for b in np.nonzero(stored)[0]:
         assert np.array_equal(kc[w.block_table[b, lens[b] // 16], :, lens[b] % 16], k_new[b])
 
 
-def test_decode_loop_is_a_fold_over_steps():
+@pytest.mark.parametrize("layout", [0, qf.QF_FLAG_KV_NHD])
+def test_decode_loop_is_a_fold_over_steps(layout):
     # Twenty decode steps: sweep the cache, fold the current token in, append it, advance.  After every step
     # the result must equal attention over all positions so far plus the current one (the appendix's fold).
     lens0 = [0, 14, 250, 1000]
@@ -177,7 +179,7 @@ def test_decode_loop_is_a_fold_over_steps():
     w = wl.make_workload("loop", cap, [wl.fixed_shards(c, 512) for c in cap], Hq, Hkv, seed=97)
     w.seq_lens = np.asarray(lens0, np.int32)
     rng = np.random.default_rng(97)
-    dw = DeviceWorkload(w)
+    dw = DeviceWorkload(w, flags=layout)
     dw.seq_lens.copy_(torch.from_numpy(w.seq_lens).cuda())
     sh = T.oracle_shape(w)
     out = torch.empty_like(dw.out)
@@ -204,8 +206,8 @@ def test_decode_loop_is_a_fold_over_steps():
         assert T.out_err(out.cpu().numpy(), ref_out) <= T.ENG_OUT, j
         assert T.lse_err(lse.cpu().numpy(), ref_lse) <= T.ENG_LSE, j
     # the device cache equals the host mirror bit for bit
-    kc = dw.k_cache.view(torch.int16).cpu().numpy().view(np.uint16)
-    assert np.array_equal(kc, w.k_cache)
+    assert np.array_equal(dw.cache_head_major("k"), w.k_cache)
+    assert np.array_equal(dw.cache_head_major("v"), w.v_cache)
 
 
 def test_decode_loop_replayed_from_one_cuda_graph():
