@@ -1,8 +1,8 @@
 /*
  * qf.h -- C ABI of the Q-First cache-side decode-attention library (B200, sm_100a).
  *
- * What the library computes (Q-First paper, Section 2 "The device needs only
- * the query" and Section 5 "The cache may be split anywhere"):
+ * What the library computes (Q-First paper, Section 2, on the device that needs
+ * only the query, and Section 5, on splitting the cache):
  *
  *   The device that holds a request's KV cache receives the query alone, one
  *   token per request, and sweeps its cached positions.  For a set S of cached
@@ -41,13 +41,17 @@
  *                       QF_FLAG_KV_NHD, token-major pages
  *                       [num_pages, page_size, Hkv, D] (the rows of one KV
  *                       head of a page are Hkv*D elements apart).  The paper
- *                       says only "paged"; both are layouts serving stacks
+ *                       only says that the cache is paged; both are layouts serving stacks
  *                       keep, and the results are the same bit for bit.
  *   block_table  int32 [B, max_pages_per_req]  logical page -> physical page.
  *                       May be NULL: then request b's logical page p is
  *                       physical page b*max_pages_per_req + p.
  *                       Entries past a request's last page are never read.
- *   seq_lens     int32 [B]          cached positions of each request
+ *   seq_lens     int32 [B]          cached positions of each request; a length
+ *                       beyond what the table row can address
+ *                       (page_size * max_pages_per_req) is treated as that
+ *                       limit (and reported as QF_STATUS_BAD_PAGE under
+ *                       QF_FLAG_CHECK_BOUNDS): the row is never overrun
  *   shard_ranges int32 [B, S, 2]    half-open token range [beg, end) of each
  *                       shard; clamped to [0, seq_lens[b]]; beg >= end after
  *                       clamping means an empty shard.  Ranges need not be
@@ -59,10 +63,15 @@
  *   out          fp32  [B, Hq, D];  lse  fp32 [B, Hq]
  *
  * Ownership: every pointer is borrowed for the duration of the enqueued work;
- * the library allocates no device memory, keeps no pointer after the work
- * completes and has no mutable global state beyond one-time per-device kernel
- * attributes and a host-side cache of TMA descriptors (1,024 entries) keyed by
- * (pointer, num_pages, num_kv_heads).  `p` is host memory, read before return.
+ * the library allocates no device memory and keeps no pointer after the work
+ * completes.  Its mutable state is: one-time per-device kernel attributes and
+ * device properties (set under a lock); a host-side cache of TMA descriptors
+ * (1,024 entries) keyed by (pointer, num_pages, num_kv_heads), also locked;
+ * the fixed QF_STATIC_SCRATCH_BYTES device array that qf_decode_partial_static
+ * uses, part of the library image on every GPU that loads it; and, per host
+ * thread, the text of the last CUDA error, the launch count of the last call
+ * and the measurement events of qf_testing.h.  `p` is host memory, read
+ * before return.
  *
  * Asynchrony: every call only enqueues work on `cuda_stream` (a cudaStream_t
  * passed as void*, NULL = the legacy default stream) and returns without
@@ -105,11 +114,7 @@ enum {
 enum {
     QF_FLAG_CHECK_BOUNDS  = 1, /* range-check page indices on the device           */
     QF_FLAG_SIMPLE_KERNEL = 2, /* use the plain-load sweep kernel (validation aid) */
-    QF_FLAG_DRAW_ALWAYS   = 8, /* default sweep kernel only: hand out the tail of the work
-                                  as drawn chunks however short the sweep is (by default
-                                  only sweeps long enough to gain from it do).  Same
-                                  results up to fp32 summation order; lets small tests
-                                  reach the drawn-chunk path                             */
+    /* 8: QF_FLAG_DRAW_ALWAYS, a test hook declared in qf_testing.h                  */
     QF_FLAG_KV_NHD        = 16 /* k_cache and v_cache are [num_pages, page_size, Hkv, D]
                                   (token-major pages) instead of [num_pages, Hkv,
                                   page_size, D]; honoured by every call that touches
@@ -213,7 +218,7 @@ int qf_combine_self(const float *o_part, const float *lse_part, const int32_t *s
                     const qf_params *p, void *cuda_stream);
 
 /*
- * Section 2, the cache write nothing waits on: stores the current token's key
+ * Section 2, the cache write (no later step of the token depends on it): stores the current token's key
  * and value (bf16 [B, Hkv, D]) at position seq_lens[b] of every request, in the
  * page block_table[b][seq_lens[b]/16] (identity table if NULL).  seq_lens is
  * not modified: the caller advances it when the next step begins.  A request
@@ -244,8 +249,8 @@ int qf_fold_append(const float *o_part, const float *lse_part, const int32_t *sh
 
 
 /*
- * Section 4 ("what each side holds": W_q and W_o live with the cache) and the
- * appendix paragraph "The cache side must batch": the projection pair at a
+ * Section 4 (placement: W_q and W_o live with the cache) and the appendix
+ * paragraph on batching at the cache side: the projection pair at a
  * layer boundary, over the co-resident requests of a batch,
  *     u' = z + W_o a              (closes the layer:  [batch, d_model])
  *     q  = W_q N_1(u')            (opens the next:    [batch, n_q])
@@ -271,7 +276,10 @@ int qf_fold_append(const float *o_part, const float *lse_part, const int32_t *sh
  * before capturing).  Meant for the paper's regime of a few co-resident
  * requests: from a batch of about 32 on a library GEMM is as fast or faster.
  * qf_project_status copies the pair's status word (QF_STATUS_TIMEOUT if a
- * bounded wait inside a kernel ran out; 0 = clean) and synchronises the stream.
+ * bounded wait inside a kernel ran out; 0 = clean), clears it and synchronises
+ * the stream.  The word is sticky: a bit raised by any pair that used this
+ * workspace (any layer of a stack, any replay of a captured graph) stays until
+ * this call has reported it once.
  */
 size_t qf_project_workspace_bytes(int batch, int d_model, int n_q);
 int qf_project_pair(const float *a, const void *z, const void *w_o, const void *g,
@@ -315,48 +323,6 @@ int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_c
 int qf_read_status(const void *workspace, int32_t *host_status, void *cuda_stream);
 
 /*
- * Diagnostic aid (no counterpart in the paper).  Every wait inside the kernels
- * is bounded: when its limit runs out the kernel records QF_STATUS_TIMEOUT and
- * returns instead of hanging.  This call enqueues a one-warp kernel that waits,
- * with a limit of a few thousand polls (under a millisecond), on a barrier that
- * nothing will ever complete, through the same wait routine; afterwards
- * qf_read_status(workspace) must report QF_STATUS_TIMEOUT and the context must
- * still be usable.  `workspace`: at least 256 bytes of device memory, 256-byte
- * aligned (its header words are overwritten).
- */
-int qf_selftest_bounded_wait(void *workspace, void *cuda_stream);
-
-/*
- * Diagnostic aid (no counterpart in the paper; host only, no GPU needed).  The
- * sweep cuts its work, `total_units` stage units of 128 tokens of one KV head,
- * into pieces: one static slice per CTA, then, for sweeps long enough (or any
- * sweep of at least two units per CTA with draw_always != 0), chunks of
- * halving size that CTAs draw from a counter.  This returns the number of
- * pieces the kernels would use for (total_units, n_ctas) and writes the first
- * min(pieces, capacity) ranges [piece_begin[p], piece_end[p]); it also checks
- * that the kernels' position-to-piece map agrees with the ranges.  Negative
- * return: QF_ERR_BAD_SHAPE (arguments out of range, or the two maps disagree),
- * QF_ERR_NULL.  n_ctas is at most 160.
- */
-int qf_plan_pieces(int total_units, int n_ctas, int draw_always, int32_t *piece_begin,
-                   int32_t *piece_end, int capacity);
-
-/*
- * Number of kernels the last qf_decode_partial / qf_combine call on this
- * thread enqueued (for launch accounting in benchmarks).
- */
-int qf_last_launch_count(void);
-
-/*
- * Measurement aid (no counterpart in the paper).  While set, every
- * qf_decode_partial on this thread records `start_event` just before and
- * `stop_event` just after its sweep kernel on the call's stream, so that a
- * benchmark can time that one kernel live.  Both are cudaEvent_t handles passed
- * as void*; pass NULL, NULL to switch it off (the default).
- */
-int qf_set_profile_events(void *start_event, void *stop_event);
-
-/*
  * The sweep for callers that cannot allocate.  (The paper has no counterpart:
  * this entry point exists for the library's users, not for the method.)
  *
@@ -384,8 +350,10 @@ int qf_set_profile_events(void *start_event, void *stop_event);
  *     word, plan, segment states), so back-to-back calls on one stream are
  *     safe; two calls whose kernels may overlap on the GPU (different streams,
  *     no ordering between them) race on the array and must not be issued.
- *   - qf_read_status cannot be pointed at the array from outside; use
- *     qf_decode_partial with QF_FLAG_CHECK_BOUNDS when a status is wanted.
+ *   - qf_read_status cannot be pointed at the array from outside:
+ *     qf_static_scratch_status reads the status word (QF_STATUS_* bits) of the
+ *     last qf_decode_partial_static on the current device and synchronises
+ *     the stream, exactly as qf_read_status does for a caller's workspace.
  * Everything else (arguments, layouts, results, error codes, asynchrony) is as
  * for qf_decode_partial.
  */
@@ -395,6 +363,8 @@ int qf_decode_partial_static(const void *q, const void *k_cache, const void *v_c
                              const int32_t *shard_ranges,
                              float *o_part, float *m_part, float *lse_part,
                              const qf_params *p, void *cuda_stream);
+
+int qf_static_scratch_status(int32_t *host_status, void *cuda_stream);
 
 /* Text describing the last QF_ERR_STATIC_SCRATCH / set-up failure on this thread. */
 const char *qf_static_scratch_error(void);

@@ -17,7 +17,8 @@
  * sharded == unsharded, pairwise fold == n-way merge, overflow cases at
  * log Z = 100, shift invariance, d(out)/d(v_j) = A_j, paging invariance,
  * SciPy / PyTorch fp64 library routines, exact-rational brute force on tiny
- * inputs.  The projection pair at the end of the file (u' = z + W_o a,
+ * inputs; the two "pick" entry points (selected outputs only) against the rows of
+ * the full set, bit for bit, and against a NumPy statement of the definition.  The projection pair at the end of the file (u' = z + W_o a,
  * q = W_q N_1(u')) has its own pins: one-hot inputs that read out weight
  * columns, exact row sums under a constant stream, power-of-two equivariance,
  * PyTorch fp64 matmul and rms_norm, exact rational brute force, nearest-bf16
@@ -342,8 +343,8 @@ int qfo_combine_fold(const double *o_part, const double *lse_part, const int32_t
 }
 
 /*
- * The accelerator-side finish of a decode step (Section 2; the fold of the
- * appendix's "what the combine is"): the cached positions act as one pseudo-token
+ * The accelerator-side finish of a decode step (Section 2; the fold stated in
+ * the appendix on the combine): the cached positions act as one pseudo-token
  * of score lse_prev and value o_prev, and the current token (k_new, v_new) is
  * appended to it:
  *     s_jj = q . k_new / sqrt(d)
@@ -389,10 +390,10 @@ int qfo_self_fold(const double *o_prev, const double *lse_prev, const uint16_t *
 
 
 /* ------------------------------------------------------------------------
- * The cache side's projection pair at a layer boundary (Section 4 "what each
- * side holds": W_q and W_o live with the cache; the stage's contract ends in
+ * The cache side's projection pair at a layer boundary (Section 4,
+ * placement: W_q and W_o live with the cache; the stage's contract ends in
  * u' = z + W_o a, and the next stage opens with q = W_q N_1(u'); the appendix
- * "The cache side must batch" makes it a product over the co-resident
+ * paragraph on batching at the cache side makes it a product over the co-resident
  * requests of a batch).
  *
  * The paper fixes bf16 weights and a bf16 residual stream (its per-layer byte

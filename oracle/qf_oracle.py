@@ -216,7 +216,7 @@ def self_fold(o_prev, lse_prev, q, k_new, v_new, sh: Shape):
 
 
 def project_pair(a, z, w_o, g, w_q, eps=1e-6, exact=False):
-    """The cache side's projection pair (Section 4; appendix "The cache side must batch"):
+    """The cache side's projection pair (Section 4; the appendix paragraph on batching at the cache side):
     u' = z + W_o a, q = W_q N_1(u') with bf16 roundings of a, u', N_1(u') and q.
     a: float32 [M, n_q]; z: bf16 bits [M, d_model]; w_o: [d_model, n_q]; g: [d_model]; w_q: [n_q, d_model].
     Returns (u bf16 bits, q bf16 bits) and, with exact=True, the fp64 values before the last rounding."""

@@ -1,5 +1,6 @@
 """Thin ctypes binding over the C ABI in ``include/qf.h``.
 
+Covers ``include/qf.h`` and the test hooks of ``include/qf_testing.h``.
 Argument marshalling only: every step of the path runs in the CUDA library.
 Functions carry the same names as the C entry points (without the ``qf_``
 prefix).  Tensor arguments may be torch tensors (their ``data_ptr()`` is
@@ -41,6 +42,7 @@ EXPORTS = (
     "qf_set_profile_events", "qf_decode_partial_static", "qf_static_scratch_error",
     "qf_combine_self", "qf_append_kv", "qf_selftest_bounded_wait", "qf_plan_pieces",
     "qf_project_workspace_bytes", "qf_project_pair", "qf_project_status", "qf_fold_append",
+    "qf_static_scratch_status", "qf_project_status_inject",
 )
 
 
@@ -109,6 +111,10 @@ def lib() -> ctypes.CDLL:
         L.qf_decode_partial_static.restype = ctypes.c_int
         L.qf_decode_partial_static.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, vp, vp, pp, vp]
         L.qf_static_scratch_error.restype = ctypes.c_char_p
+        L.qf_static_scratch_status.restype = ctypes.c_int
+        L.qf_static_scratch_status.argtypes = [ctypes.POINTER(ctypes.c_int32), vp]
+        L.qf_project_status_inject.restype = ctypes.c_int
+        L.qf_project_status_inject.argtypes = [vp, ctypes.c_int32, vp]
         L.qf_fold_append.restype = ctypes.c_int
         L.qf_fold_append.argtypes = [vp, vp, i32p, vp, vp, vp, vp, vp, vp, vp, i32p, i32p, ctypes.c_int, pp, vp]
         L.qf_project_workspace_bytes.restype = ctypes.c_size_t
@@ -197,6 +203,22 @@ def decode_partial_static(q, k_cache, v_cache, block_table, seq_lens, shard_rang
         detail = lib().qf_static_scratch_error().decode()
         raise QFError(rc, "qf_decode_partial_static" + (f" ({detail})" if detail else ""))
     return rc
+
+
+def static_scratch_status(stream=None) -> int:
+    """Status bits of the last decode_partial_static on the current device (synchronises the stream)."""
+    st = ctypes.c_int32(0)
+    rc = lib().qf_static_scratch_status(ctypes.byref(st), _stream(stream))
+    if rc != QF_OK:
+        raise QFError(rc, "qf_static_scratch_status")
+    return int(st.value)
+
+
+def project_status_inject(workspace, bits: int, stream=None) -> None:
+    """Test hook: OR status bits into the projection pair's status word as a timed-out kernel would."""
+    rc = lib().qf_project_status_inject(_ptr(workspace), int(bits), _stream(stream))
+    if rc != QF_OK:
+        raise QFError(rc, "qf_project_status_inject")
 
 
 def combine(o_part, lse_part, shard_counts, out, lse, p: QFParams, stream=None, check: bool = True) -> int:

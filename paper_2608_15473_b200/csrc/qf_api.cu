@@ -8,6 +8,7 @@
 #include <cstring>
 
 #include "../../include/qf.h"
+#include "../../include/qf_testing.h"
 #include "qf_combine.cuh"
 #include "qf_common.cuh"
 #include "qf_proj.cuh"
@@ -43,6 +44,7 @@ int validate(const qf_params *p)
     if (p->batch > 65535 || p->num_kv_heads > 65535) return QF_ERR_UNSUPPORTED;
     if ((long long)p->batch * p->max_shards * p->num_kv_heads > (1ll << 22)) return QF_ERR_UNSUPPORTED;
     if ((long long)p->num_pages * p->num_kv_heads * qf::kPageSize >= (1ll << 31)) return QF_ERR_UNSUPPORTED;
+    if ((long long)p->max_pages_per_req * qf::kPageSize >= (1ll << 31)) return QF_ERR_UNSUPPORTED;
     return QF_OK;
 }
 
@@ -65,9 +67,11 @@ qf::DevParams dev_params(const qf_params *p)
     return d;
 }
 
-// One-time check per device that this is a compute-capability 10.x part.
+// One-time check per device that this is a compute-capability 10.x part (cached under a lock: any host
+// thread may be the first to use a device).
 int check_device(int *sm_count)
 {
+    static std::mutex mu;
     static int cached_major[64];
     static int cached_sms[64];
     static bool known[64];
@@ -75,6 +79,7 @@ int check_device(int *sm_count)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
     if (dev < 0 || dev >= 64) return QF_ERR_DEVICE;
+    std::lock_guard<std::mutex> lock(mu);
     if (!known[dev]) {
         int major = 0, sms = 0;
         e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
@@ -421,7 +426,7 @@ int qf_project_pair(const float *a, const void *z, const void *w_o, const void *
     const int sb_q = qf::proj_ring(d_model / (qf::kProjSplits * qf::kProjBoxK), np).sb;
     if (qf::make_weight_map(&map_o, w_o, d_model, n_q, sb_o, g_cuda_msg, sizeof g_cuda_msg)) return QF_ERR_CUDA;
     if (qf::make_weight_map(&map_q, w_q, n_q, d_model, sb_q, g_cuda_msg, sizeof g_cuda_msg)) return QF_ERR_CUDA;
-    unsigned *status = (unsigned *)workspace;
+    unsigned long long *status = (unsigned long long *)workspace;
     float *ssq_part = (float *)((char *)workspace + 256);
 
     qf::ProjArgs s0 = {};
@@ -442,13 +447,33 @@ int qf_project_pair(const float *a, const void *z, const void *w_o, const void *
 int qf_project_status(const void *workspace, int32_t *host_status, void *cuda_stream)
 {
     if (!workspace || !host_status) return QF_ERR_NULL;
-    unsigned word = 0;
+    unsigned long long word = 0;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     cudaError_t e = cudaMemcpyAsync(&word, workspace, sizeof word, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync");
+    // read and clear: the bits are sticky until somebody has seen them (an untagged word reads as clean)
+    e = cudaMemsetAsync(const_cast<void *>(workspace), 0, sizeof word, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
-    *host_status = (int32_t)word;
+    *host_status = ((word >> 8) == qf::kProjStatusTag) ? (int32_t)(word & 0xffull) : 0;
+    return QF_OK;
+}
+
+namespace {
+__global__ void proj_status_inject_kernel(unsigned long long *w, unsigned bits) { qf::proj_status_or(w, bits); }
+}  // namespace
+
+int qf_project_status_inject(void *workspace, int32_t bits, void *cuda_stream)
+{
+    if (!workspace) return QF_ERR_NULL;
+    if ((uintptr_t)workspace & 255) return QF_ERR_WORKSPACE;
+    int rc = check_device(nullptr);
+    if (rc != QF_OK) return rc;
+    proj_status_inject_kernel<<<1, 1, 0, (cudaStream_t)cuda_stream>>>((unsigned long long *)workspace,
+                                                                      (unsigned)bits & 0xffu);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "proj_status_inject_kernel launch");
     return QF_OK;
 }
 

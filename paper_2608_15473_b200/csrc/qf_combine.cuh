@@ -135,7 +135,7 @@ combine_kernel(const float *__restrict__ o_part, const float *__restrict__ lse_p
                                 sm_scale);
 }
 
-// The cache write nothing waits on (Section 2): the current token's key and value go to position
+// The cache write of Section 2 (no later step of the token depends on it): the current token's key and value go to position
 // seq_lens[b] of request b, through the block table.  One warp per (request, KV head).
 // Physical page of position pos of request b, or -1 if the request has no page for it.
 __device__ __forceinline__ long long append_page(const int *__restrict__ block_table, int b, int pos, const DevParams &P)

@@ -172,13 +172,16 @@ __device__ __forceinline__ size_t out_entry(const DevParams &P, int e)
     return (size_t)b * P.out_shards + P.out_shard0 + s;
 }
 
-// Clamp a shard's token range to the request's cached length.
-__device__ __forceinline__ void clamp_range(int r0, int r1, int len, int &beg, int &end)
+// Clamp a shard's token range to the request's cached length, and the length to what the request's
+// block-table row can address (max_tokens = 16 * max_pages_per_req): a length beyond the row is a caller
+// error, and the sweep must not follow it past the row.
+__device__ __forceinline__ void clamp_range(int r0, int r1, int len, int max_tokens, int &beg, int &end)
 {
     beg = max(r0, 0);
-    end = min(r1, len);
+    end = min(r1, min(len, max_tokens));
     if (end < beg) end = beg;
 }
+__host__ __device__ __forceinline__ int max_row_tokens(int max_pages_per_req) { return max_pages_per_req * kPageSize; }
 
 // Launch with the programmatic-stream-serialization attribute (see grid_dependency_wait).
 template <typename... KArgs, typename... Args>

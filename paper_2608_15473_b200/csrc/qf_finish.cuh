@@ -1,4 +1,4 @@
-// The finish kernel of the cache-side sweep (Section 5: partial states "merged in any order"): merges the
+// The finish kernel of the cache-side sweep (Section 5: partial states are order-independent): merges the
 // (shard, KV head) units that the sweep's piece boundaries cut into segments.
 #pragma once
 

@@ -1,6 +1,6 @@
 // The cache side's projection pair at a layer boundary (Section 4: the cache side holds W_q and W_o;
-// a stage ends in u' = z + W_o a and the next one opens with q = W_q N_1(u'); appendix "The cache side
-// must batch": the products run over the co-resident requests of a batch).
+// a stage ends in u' = z + W_o a and the next one opens with q = W_q N_1(u'); the appendix paragraph on
+// batching at the cache side: the products run over the co-resident requests of a batch).
 //
 // Both products are skinny: a few requests (at most 64 here) against a weight matrix of tens of
 // megabytes that is read exactly once.  They are bound by streaming the weight, so the kernel is built
@@ -63,13 +63,29 @@ struct ProjArgs {
     const uint16_t *z;         // stage 0: [batch][n_out] bf16
     uint16_t *out;             // [batch][n_out] bf16 (u' or q)
     float *ssq_part;           // [tiles of stage 0][kProjMaxBatch]: stage 0 writes, stage 1 reads
-    unsigned *status;          // bit 1 (QF_STATUS_TIMEOUT) is ORed in when a wait runs out
+    unsigned long long *status; // tagged status word (proj_status_or): QF_STATUS_TIMEOUT is ORed in when a wait runs out
     int batch, n_out, k_total;
     int ssq_tiles;             // stage 1: number of stage 0 tiles
     int ring_sb, ring_slots;   // boxes per TMA request, requests in flight per CTA (proj_ring)
     int recv_aliased;          // the split-K receive area reuses the ring (large batches) instead of its own room
     float inv_d_model, eps;    // stage 1
 };
+
+// The pair's status word is STICKY: bits stay until the host reads them (qf_project_status reads and clears),
+// so a failure in one layer's pair is not wiped by the next layer's, nor by a later replay of a captured graph.
+// The workspace is never assumed initialised: a word counts only if its upper 56 bits carry this tag, anything
+// else reads as "clean".
+constexpr unsigned long long kProjStatusTag = 0x51F1A7C0DE5EEDull;   // 56 bits
+__device__ __forceinline__ void proj_status_or(unsigned long long *w, unsigned bits)
+{
+    unsigned long long old = *reinterpret_cast<volatile unsigned long long *>(w);
+    for (int tries = 0; tries < (1 << 12); ++tries) {
+        const unsigned long long cur = ((old >> 8) == kProjStatusTag) ? (old & 0xffull) : 0ull;
+        const unsigned long long prev = atomicCAS(w, old, (kProjStatusTag << 8) | cur | bits);
+        if (prev == old) return;
+        old = prev;
+    }
+}
 
 // ---- tcgen05 / cluster PTX
 __device__ __forceinline__ void tmem_alloc(uint32_t holder_smem, uint32_t ncols)
@@ -259,7 +275,6 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
 
     grid_dependency_wait();     // everything below reads what earlier kernels of the stream wrote
     grid_launch_dependents();
-    if (STAGE == 0 && blockIdx.x == 0 && tid == 0) *A.status = 0u;
 
     // ---- activations of this K slice, as the B operand: [NP rows][k_slice] bf16, 128B-swizzled boxes.
     // Global loads are issued eight items at a time per thread before any of them is used (the prologue is
@@ -416,7 +431,7 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
             umma_commit(smem_u32(&sm.mma_done));
         } else {
             sm.abort_flag = 1;
-            atomicOr(A.status, (unsigned)kStatusTimeout);
+            proj_status_or(A.status, (unsigned)kStatusTimeout);
             // copies still in flight must land before this CTA's shared memory goes away
             for (int r = consumed; r < issued; ++r)
                 for (unsigned it = 0; it < (1u << 20); ++it)
@@ -430,7 +445,7 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
         return;
     }
     const bool done = mbar_wait(smem_u32(&sm.mma_done), 0, abort_flag) && !*abort_flag;
-    if (!done && tid == 0) { sm.abort_flag = 1; atomicOr(A.status, (unsigned)kStatusTimeout); }
+    if (!done && tid == 0) { sm.abort_flag = 1; proj_status_or(A.status, (unsigned)kStatusTimeout); }
     tc_fence_after();
 
     // ---- split-K sum.  Rank r finishes requests n = 8 i + r (all 128 features of each): every rank sends
@@ -473,7 +488,7 @@ proj_kernel(const __grid_constant__ CUtensorMap w_map, ProjArgs A)
             landed = mbar_try_wait(smem_u32(&sm.recv_full), 0u);
             if (!landed && it > 64) __nanosleep(64);
         }
-        if (!landed && tid == 0) atomicOr(A.status, (unsigned)kStatusTimeout);
+        if (!landed && tid == 0) proj_status_or(A.status, (unsigned)kStatusTimeout);
     }
 
     // ---- the eight partials of this rank's requests, summed in rank order, and the epilogue
@@ -600,14 +615,18 @@ cudaError_t launch_proj_np(const CUtensorMap &map, const ProjArgs &args, cudaStr
     a2.recv_aliased = ring.own_recv ? 0 : 1;
     const size_t smem = proj_smem_bytes(ring.sb * ring.slots, n_boxes, NP, ring.own_recv);
     // the attribute is raised once per device to the largest footprint this instantiation can have
-    static bool attr_set[64];
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (!attr_set[dev & 63]) {
-        cudaError_t ea = cudaFuncSetAttribute(proj_kernel<STAGE, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              227 * 1024);
-        if (ea != cudaSuccess) return ea;
-        attr_set[dev & 63] = true;
+    {
+        static std::mutex attr_mu;   // any host thread may be the first on a device
+        static bool attr_set[64];
+        int dev = 0;
+        cudaGetDevice(&dev);
+        std::lock_guard<std::mutex> lock(attr_mu);
+        if (!attr_set[dev & 63]) {
+            cudaError_t ea = cudaFuncSetAttribute(proj_kernel<STAGE, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                  227 * 1024);
+            if (ea != cudaSuccess) return ea;
+            attr_set[dev & 63] = true;
+        }
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(args.n_out / kProjTileOut * kProjSplits));

@@ -98,10 +98,10 @@ inline WorkspaceLayout workspace_layout(int batch, int max_shards, int num_kv_he
 // Work units of entry e = (request, shard), all KV heads together: stage units of kPagesPerStage pages
 // per KV head.
 __device__ __forceinline__ int entry_units(const int *__restrict__ seq_lens, const int *__restrict__ shard_ranges,
-                                           int e, int max_shards, int num_kv_heads)
+                                           int e, int max_shards, int num_kv_heads, int max_tokens)
 {
     int beg, end;
-    clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[e / max_shards], beg, end);
+    clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[e / max_shards], max_tokens, beg, end);
     if (end <= beg) return 0;
     const int npages = ((end - 1) >> 4) - (beg >> 4) + 1;
     return ((npages + kPagesPerStage - 1) / kPagesPerStage) * num_kv_heads;
@@ -185,14 +185,14 @@ __host__ __device__ __forceinline__ void piece_range(const PieceGrid &g, int n_c
 // prefix[e] = number of stage units before entry e = b*S + s, left in scratch.
 __global__ void __launch_bounds__(1024)
 plan_kernel(const int *__restrict__ seq_lens, const int *__restrict__ shard_ranges, int *__restrict__ prefix,
-            int n_entries, int max_shards, int num_kv_heads)
+            int n_entries, int max_shards, int num_kv_heads, int max_tokens)
 {
     __shared__ int warp_sums[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int carry = 0;
     for (int base = 0; base < n_entries; base += 1024) {
         const int e = base + tid;
-        const int cnt = (e < n_entries) ? entry_units(seq_lens, shard_ranges, e, max_shards, num_kv_heads) : 0;
+        const int cnt = (e < n_entries) ? entry_units(seq_lens, shard_ranges, e, max_shards, num_kv_heads, max_tokens) : 0;
         int x = cnt;  // inclusive scan within the warp
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -264,6 +264,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = P.max_shards, Hkv = P.num_kv_heads, Hq = P.num_q_heads;
     const int n_entries = P.batch * S;
+    const int max_tokens = max_row_tokens(P.max_pages_per_req);
     volatile int *abort_flag = &sm.abort_flag;
 
     if (tid == 0) {
@@ -297,7 +298,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
         for (int base = 0; base < n_entries; base += kConsumerThreads) {
             const int e = base + tid;
             const int cnt = (tid < kConsumerThreads && e < n_entries)
-                                ? entry_units(seq_lens, shard_ranges, e, S, Hkv) : 0;
+                                ? entry_units(seq_lens, shard_ranges, e, S, Hkv, max_tokens) : 0;
             int x = cnt;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
@@ -322,6 +323,11 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
         prefix = sm.prefix;
     }
     const unsigned long long epoch = sm.epoch;   // written before the plan's barriers
+    if (P.check_bounds && blockIdx.x == 0) {
+        // a cached length that the request's block-table row cannot address was clamped by the plan: report it
+        for (int b = tid; b < P.batch; b += kSweepThreads)
+            if (seq_lens[b] > max_tokens) epoch_or(header + kHdrStatus, epoch, kStatusBadPage);
+    }
     const int total = prefix[n_entries];
     const int n_ctas = (int)gridDim.x;
     // a prefix left in global memory (very large batches) makes locating a piece's first entry slow: static only
@@ -378,8 +384,8 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                 const int seg_len = min(nunits - j, pos1 - pos);
                 const int b = e / S;
                 if (e != cur_e) {
-                    if (e == nxt_e) clamp_range(nxt_r0, nxt_r1, nxt_len, beg, end);
-                    else clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[b], beg, end);
+                    if (e == nxt_e) clamp_range(nxt_r0, nxt_r1, nxt_len, max_tokens, beg, end);
+                    else clamp_range(shard_ranges[2 * e], shard_ranges[2 * e + 1], seq_lens[b], max_tokens, beg, end);
                     cur_e = e;
                     if (e == nxt_tbl_e) { head_tbl = nxt_tbl; head_tbl_e = e; }
                     // start fetching the next non-empty shard's range; it is consumed a segment later
@@ -420,7 +426,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
                     if (u == 1 && nxt_e >= 0 && nxt_tbl_e != nxt_e) {
                         // the next shard's range has arrived by now: fetch its first table entries too
                         int nb, ne;
-                        clamp_range(nxt_r0, nxt_r1, nxt_len, nb, ne);
+                        clamp_range(nxt_r0, nxt_r1, nxt_len, max_tokens, nb, ne);
                         nxt_tbl = load_tbl(nxt_e / S, nb >> 4, (ne - 1) >> 4);
                         nxt_tbl_e = nxt_e;
                     }
@@ -745,18 +751,23 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
     float *seg = reinterpret_cast<float *>(ws + wsl.seg_off);
     const int n_entries = P.batch * P.max_shards;
     const size_t smem = sizeof(SweepSmem<G>) + 1024;
-    static bool attr_set[64];
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (!attr_set[dev & 63]) {
-        cudaError_t e = cudaFuncSetAttribute(sweep_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) { snprintf(msg, msg_len, "cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return -5; }
-        attr_set[dev & 63] = true;
+    {   // per-device kernel attribute, set once under a lock (any host thread may come first)
+        static std::mutex attr_mu;
+        static bool attr_set[64];
+        int dev = 0;
+        cudaGetDevice(&dev);
+        std::lock_guard<std::mutex> lock(attr_mu);
+        if (!attr_set[dev & 63]) {
+            cudaError_t e = cudaFuncSetAttribute(sweep_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) { snprintf(msg, msg_len, "cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return -5; }
+            attr_set[dev & 63] = true;
+        }
     }
     *launches = 0;
     const int *global_prefix = nullptr;
     if (n_entries > kMaxSmemEntries) {
-        plan_kernel<<<1, 1024, 0, st>>>(sl, sr, prefix, n_entries, P.max_shards, P.num_kv_heads);
+        plan_kernel<<<1, 1024, 0, st>>>(sl, sr, prefix, n_entries, P.max_shards, P.num_kv_heads,
+                                        max_row_tokens(P.max_pages_per_req));
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) { snprintf(msg, msg_len, "plan_kernel launch: %s", cudaGetErrorString(e)); return -5; }
         global_prefix = prefix;

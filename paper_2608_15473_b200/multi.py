@@ -37,7 +37,7 @@ def whole_job_throughput(total_bytes: float, max_ms_per_step: float) -> float:
 # the same exchange needs no collective at all: with out_shards / out_shard_offset in the parameters
 # (rank_sweep_params) every rank's qf_decode_partial writes its slots of the OWNER's [B, S, Hq, D] arrays,
 # passed as peer-mapped pointers; the sweep kernel writes shard states with plain stores, so its epilogue
-# is the transfer ("parked, not pushed"), and the owner merges after a barrier.
+# is the transfer (Section 3: results are left where the other side reads them), and the owner merges after a barrier.
 # --------------------------------------------------------------------------------------------------
 def shard_slice(max_shards: int, world_size: int, rank: int) -> range:
     """Shard slots [lo, hi) of every request that ``rank`` sweeps: equal blocks of ceil(S/world)."""

@@ -18,7 +18,7 @@ def built():
 
 
 def declared_functions():
-    text = (ROOT / "include" / "qf.h").read_text()
+    text = "".join(h.read_text() for h in sorted((ROOT / "include").glob("*.h")))
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(qf_[a-z_]+)\s*\(", text)))
 
@@ -114,3 +114,16 @@ def test_no_device_is_a_loud_error_not_a_fallback():
         from paper_2608_15473_b200.runtime import DeviceWorkload
         from paper_2608_15473_b200 import workloads as wl
         DeviceWorkload(wl.make_workload("x", [16], [[(0, 16)]], 2, 1))
+
+
+def test_static_scratch_entry_rejects_without_touching_a_device():
+    # invalid parameters and over-large problems are turned away before any device call
+    p = good()
+    p.head_dim = 64
+    a = 0x10000
+    assert qf.decode_partial_static(a, a, a, None, a, a, a, a, a, p, stream=0, check=False) == qf.QF_ERR_UNSUPPORTED
+    p = good()
+    p.batch = 0
+    assert qf.decode_partial_static(a, a, a, None, a, a, a, a, a, p, stream=0, check=False) == qf.QF_ERR_BAD_SHAPE
+    big = qf.params(batch=4096, num_q_heads=32, num_kv_heads=8, max_pages_per_req=64, max_shards=8, num_pages=1 << 18)
+    assert qf.decode_partial_static(a, a, a, None, a, a, a, a, a, big, stream=0, check=False) == qf.QF_ERR_STATIC_SCRATCH

@@ -483,3 +483,84 @@ def test_self_fold_large_magnitudes():
     assert abs(s_self[0, 0] - 100.0) < 0.05
     assert lse[0, 0] == pytest.approx(np.logaddexp(100.0, s_self[0, 0]), rel=1e-15) and np.isfinite(out).all()
     assert abs(out[0, 0, 1] - 1.0) < 0.02   # about half of v = 2 in the channels where o_prev is 0
+
+
+# ---------------------------------------------------------------- the "pick" entry points
+def _pick_workload():
+    # ragged lengths; shards that are clamped at both ends, empty, unaligned, overlapping, past the end;
+    # a shuffled table with spare pool pages and NaN in everything that must not be read
+    lens = [100, 0, 37, 300, 16, 1, 129]
+    ranges = [
+        [(0, 7), (7, 7), (7, 33), (33, 100)],
+        [(0, 0), (0, 5), (3, 2), (0, 0)],
+        [(0, 500), (-5, 10), (36, 37), (40, 50)],
+        [(0, 128), (128, 129), (129, 257), (250, 300)],
+        [(0, 16), (16, 16), (5, 11), (0, 0)],
+        [(0, 1), (1, 1), (0, 0), (-3, 9)],
+        [(17, 95), (1, 129), (128, 129), (64, 64)],
+    ]
+    return wl.make_workload("pick", lens, ranges, 12, 4, seed=71, pool_factor=1.4, poison_unused=True,
+                            poison_tails=True, max_pages_per_req=24)
+
+
+def test_picked_shard_states_equal_the_rows_of_the_full_set():
+    # qfo_decode_partial_pick is what the full-size GPU checks compare against: a wrong stride on the
+    # (b, s, h) triples, a missed clamp or a wrong output row would show here
+    w = _pick_workload()
+    sh = shape_of(w)
+    op, mp, lp = partials(w)
+    rng = np.random.default_rng(5)
+    B, S, H = w.batch, w.max_shards, w.num_q_heads
+    every = [(b, s, h) for b in range(B) for s in range(S) for h in range(H)]
+    order = rng.permutation(len(every))
+    pick = [every[i] for i in order] + [every[i] for i in rng.integers(len(every), size=40)]   # shuffled, with repeats
+    o, m, l = orc.decode_partial_pick(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.shard_ranges, sh, pick)
+    pk = np.asarray(pick)
+    assert np.array_equal(o, op[pk[:, 0], pk[:, 1], pk[:, 2]])
+    assert np.array_equal(m, mp[pk[:, 0], pk[:, 1], pk[:, 2]], equal_nan=False)
+    assert np.array_equal(l, lp[pk[:, 0], pk[:, 1], pk[:, 2]], equal_nan=False)
+    # a single triple, and the same triple three times
+    one = orc.decode_partial_pick(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.shard_ranges, sh, [(3, 2, 7)])
+    assert np.array_equal(one[0][0], op[3, 2, 7]) and one[2][0] == lp[3, 2, 7]
+    rep = orc.decode_partial_pick(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.shard_ranges, sh,
+                                  [(6, 1, 11)] * 3)
+    assert all(np.array_equal(rep[0][i], op[6, 1, 11]) for i in range(3))
+
+
+def test_picked_shard_states_against_numpy_definition():
+    # not only against the oracle's other entry point: a few triples written out with NumPy from the
+    # definition (scores through the table, clamped range, softmax, weighted mean of the value rows)
+    w = _pick_workload()
+    sh = shape_of(w)
+    pick = [(0, 2, 5), (2, 0, 0), (3, 3, 11), (6, 0, 9), (2, 1, 4), (5, 3, 2)]
+    o, m, l = orc.decode_partial_pick(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.shard_ranges, sh, pick)
+    G = w.group
+    for i, (b, s, h) in enumerate(pick):
+        L = int(w.seq_lens[b])
+        lo, hi = (int(x) for x in w.shard_ranges[b, s])
+        lo, hi = max(lo, 0), min(hi, L)
+        K = token_rows(w, w.k_cache, b, h // G)[lo:hi]
+        V = token_rows(w, w.v_cache, b, h // G)[lo:hi]
+        sc = K @ wl.bf16_bits_to_f64(w.q[b, h]) / math.sqrt(128.0)
+        assert len(sc) > 0
+        p = np.exp(sc - sc.max())
+        assert m[i] == pytest.approx(sc.max(), rel=1e-14)
+        assert l[i] == pytest.approx(sc.max() + math.log(p.sum()), rel=1e-13)
+        assert np.allclose(o[i], (p[:, None] * V).sum(0) / p.sum(), rtol=1e-12, atol=1e-14)
+
+
+def test_picked_unsharded_results_equal_the_rows_of_the_full_set():
+    w = _pick_workload()
+    sh = shape_of(w)
+    out, lse = full(w)
+    rng = np.random.default_rng(6)
+    B, H = w.batch, w.num_q_heads
+    every = [(b, h) for b in range(B) for h in range(H)]
+    pick = [every[i] for i in rng.permutation(len(every))] + [every[i] for i in rng.integers(len(every), size=25)]
+    o, l = orc.decode_full(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, sh, pick=pick)
+    pk = np.asarray(pick)
+    assert np.array_equal(o, out[pk[:, 0], pk[:, 1]])
+    assert np.array_equal(l, lse[pk[:, 0], pk[:, 1]])
+    assert np.isneginf(l[pk[:, 0] == 1]).all() and (o[pk[:, 0] == 1] == 0).all()     # the empty request
+    one_o, one_l = orc.decode_full(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, sh, pick=[(6, 10)])
+    assert np.array_equal(one_o[0], out[6, 10]) and one_l[0] == lse[6, 10]

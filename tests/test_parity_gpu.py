@@ -374,15 +374,63 @@ def test_host_step_matches_device_path(pinned):
     assert np.array_equal(hs.lse_host.numpy().astype(np.float64), lse)
 
 
-# T8: the benchmark configurations at full size, sampled outputs
-@pytest.mark.parametrize("cfg,seed,flags", [(2, 0, 0), (3, 0, 0), (4, 0, 0), (5, 0, 0), (2, 1, 0), (2, 2, 0), (3, 1, 0),
-                                            (3, 2, 0), (4, 1, 0), (3, 0, qf.QF_FLAG_KV_NHD), (2, 0, qf.QF_FLAG_KV_NHD)])
-def test_full_size_configs_sampled(cfg, seed, flags):
+# T8: the five benchmark configurations x seeds 0-2 at full size, in the launch configuration the benchmark
+# times, EVERY element of every output: shard states against the oracle's shard states, merged results against
+# the oracle's unsharded sweep.  (The oracle finishes the largest of them in seconds on the host cores.)
+@pytest.mark.parametrize("seed", [0, 1, 2])
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_full_size_configs_every_element(cfg, seed):
     w = wl.CONFIGS[cfg](seed=seed)
+    assert T.covers_context(w)
+    dw = run(w)
+    errs = T.compare_all(dw, w, tag=w.name)
+    print(w.name, seed, errs)
+    assert dw.status() == 0
+    # unused shard slots follow the empty convention
+    got_op, got_mp, got_lp, _, _ = dw.results()
+    for b in range(w.batch):
+        n = int(w.shard_counts[b])
+        assert np.isneginf(got_lp[b, n:]).all() and np.isneginf(got_mp[b, n:]).all() and (got_op[b, n:] == 0).all()
+
+
+# the same at full size for the variants off the headline: the one-million-token request behind a shuffled
+# table, and token-major pages; every element again
+@pytest.mark.parametrize("cfg,kwargs,flags", [(4, dict(table="shuffled"), 0), (3, {}, qf.QF_FLAG_KV_NHD),
+                                              (2, {}, qf.QF_FLAG_KV_NHD), (4, {}, qf.QF_FLAG_KV_NHD)])
+def test_full_size_variants_every_element(cfg, kwargs, flags):
+    w = wl.CONFIGS[cfg](seed=0, **kwargs)
     dw = run(w, flags)
-    errs = T.compare_sampled(dw, w, seed=cfg + 10 * seed, tag=w.name)
+    T.compare_all(dw, w, tag=f"{w.name} {kwargs} flags={flags}")
+    assert dw.status() == 0
+
+
+# sampled outputs, computed one by one by the oracle's pick entry points (pinned on the CPU against the full
+# set): the fast form of the check above, kept for the largest configuration under a second seed family
+def test_full_size_config_sampled():
+    w = wl.config5(seed=7)
+    dw = run(w)
+    errs = T.compare_sampled(dw, w, seed=57, tag=w.name)
     print(w.name, errs)
     assert dw.status() == 0
+
+
+# A cached length beyond what the request's block-table row can address (a caller error) is treated as the row's
+# limit: the sweep never indexes past the row (the entries after it belong to the next request).  With the
+# bounds flag it is also reported.
+@pytest.mark.parametrize("flags", KERNELS)
+def test_length_beyond_the_table_row_is_clamped_and_reported(flags):
+    flags, Hkv = flags
+    mp = 8                                   # 128 tokens per row
+    lens = [128, 100, 64]
+    w = wl.make_workload("overlong", lens, [[(0, 500), (60, 2000)], [(0, 100), (0, 0)], [(0, 64), (10, 20)]],
+                         2 * Hkv, Hkv, seed=37, max_pages_per_req=mp, poison_tails=True)
+    for chk in (0, qf.QF_FLAG_CHECK_BOUNDS):
+        dw = DeviceWorkload(w, flags=flags | chk)
+        dw.seq_lens.copy_(torch.tensor([200, 100, 64], dtype=torch.int32))   # request 0 claims 200 > 8 * 16
+        dw.poison_outputs()
+        dw.step()
+        T.compare_all(dw, w, tag=f"check={chk}")          # the oracle sees the honest length, 128
+        assert dw.status() == (qf.QF_STATUS_BAD_PAGE if chk else 0)
 
 
 @pytest.mark.parametrize("Hkv,flags", [(2, 0), (8, 0), (8, qf.QF_FLAG_DRAW_ALWAYS)])

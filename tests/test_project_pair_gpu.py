@@ -241,3 +241,67 @@ def test_random_shapes(seed):
     u, q, _ = run_gpu(a, z, w_o, g, w_q, 1e-6)
     ref_u, ref_q = orc.project_pair(a, z, w_o, g, w_q, eps=1e-6)
     check(u, q, ref_u, ref_q, f"seed={seed} batch={batch} d_model={d_model} n_q={n_q}")
+
+
+@pytest.mark.parametrize("batch,d_model,n_q", [(8, 1024, 2048), (8, 2560, 4096), (40, 2560, 4096)])
+def test_against_the_values_before_the_last_rounding(batch, d_model, n_q):
+    # Not through shared rounding points: the oracle also returns u' and q BEFORE their last rounding
+    # (fp64 sums of exact products).  A correctly rounded result lies within half a bf16 unit of that value;
+    # the kernel's fp32 accumulation adds a few 1e-7 of the row's scale on top (K terms of relative error
+    # 2^-24 each, random signs: sqrt(K) 2^-24 of the terms' scale, taken as 4e-6 of the row's rms here).
+    # For q the exact value is a function of the oracle's OWN rounded stream, and a flipped u' element on the
+    # GPU side moves a whole row of q by up to 1e-3 of its scale (see the module docstring): that term stays.
+    a, z, w_o, g, w_q = make_inputs(batch, d_model, n_q, seed=batch + 3 * d_model)
+    u, q, _ = run_gpu(a, z, w_o, g, w_q, 1e-6)
+    _, _, u_exact, q_exact = orc.project_pair(a, z, w_o, g, w_q, eps=1e-6, exact=True)
+    for name, got, exact, abs_tol in (("u'", u, u_exact, 4e-6), ("q", q, q_exact, 2.5e-3)):
+        x = bits_to_f64(got)
+        rms = np.sqrt((exact ** 2).mean(axis=1, keepdims=True))
+        d = np.abs(x - exact)
+        lim = 0.5 * ulp_bf16(np.maximum(np.abs(exact), np.abs(x))) + abs_tol * rms
+        worst = np.unravel_index(np.argmax(d - lim), d.shape)
+        assert (d <= lim).all(), (name, "at", worst, "got", x[worst], "exact", exact[worst], "limit", lim[worst])
+
+
+def test_against_the_chain_without_any_intermediate_rounding():
+    # The definition itself, with NumPy in fp64 and NO rounding of a, u', N_1(u') or q: what the pair computes
+    # up to the bf16 roundings the stream's dtype forces.  Each rounding is a relative error of at most 2^-9 per
+    # element with random sign, so a row of q is off by well under one percent of its scale in the mean, and no
+    # element by more than a few percent; a misplaced or missing step (gain, residual, normalisation, eps, a
+    # transposed weight) would be off by tens of percent.
+    batch, d_model, n_q = 8, 2560, 4096
+    a, z, w_o, g, w_q = make_inputs(batch, d_model, n_q, seed=123)
+    eps = 1e-6
+    u, q, _ = run_gpu(a, z, w_o, g, w_q, eps)
+    Wo, Wq, gg, zz = bits_to_f64(w_o), bits_to_f64(w_q), bits_to_f64(g), bits_to_f64(z)
+    u_true = zz + a.astype(np.float64) @ Wo.T
+    x_true = gg * u_true / np.sqrt((u_true ** 2).mean(axis=1, keepdims=True) + eps)
+    q_true = x_true @ Wq.T
+    for name, got, true, mean_tol, max_tol in (("u'", u, u_true, 3e-3, 2e-2), ("q", q, q_true, 6e-3, 4e-2)):
+        x = bits_to_f64(got)
+        rms = np.sqrt((true ** 2).mean(axis=1, keepdims=True))
+        rel = np.abs(x - true) / rms
+        assert np.sqrt((rel ** 2).mean()) < mean_tol and rel.max() < max_tol, (name, np.sqrt((rel ** 2).mean()), rel.max())
+
+
+def test_status_word_is_sticky_until_it_is_read():
+    # a timeout raised by one layer's pair must survive the pairs of the layers after it (they share the
+    # workspace) until the host reads it; reading clears it.  The failure is made on the host: the test hook
+    # ORs the bit in exactly as a kernel whose bounded wait ran out would; no kernel waits on anything.
+    batch, d_model, n_q = 8, 1024, 2048
+    a, z, w_o, g, w_q = make_inputs(batch, d_model, n_q, seed=9)
+    u, q, args = run_gpu(a, z, w_o, g, w_q, 1e-6)
+    ws = args[-1]
+    assert qf.project_status(ws) == 0
+    qf.project_status_inject(ws, qf.QF_STATUS_TIMEOUT)
+    for _ in range(5):                      # "layers 1 to L-1"
+        qf.project_pair(*args)
+    assert qf.project_status(ws) == qf.QF_STATUS_TIMEOUT
+    assert qf.project_status(ws) == 0       # read once, then clean
+    qf.project_pair(*args)
+    torch.cuda.synchronize()
+    assert qf.project_status(ws) == 0
+    assert np.array_equal(host_bits(args[5]), u) and np.array_equal(host_bits(args[6]), q)
+    # an uninitialised workspace (any bit pattern without the tag) reads as clean
+    ws.fill_(0xA5)
+    assert qf.project_status(ws) == 0
