@@ -464,6 +464,96 @@ def small_request_latency(args, qf, wl, DeviceWorkload, device, stream, barrier,
     return rec
 
 
+def run_split_request(args, dist, rank, world, local_rank, device):
+    """--split-request: ONE request's cache (the one-million-token workload, 16 shards) split over the N ranks.
+    Every rank draws the same seeded workload on its host and uploads only the pages of the shards it owns; a
+    step is query broadcast -> every rank's sweep into the owner's shard-state arrays (peer-mapped, plain stores)
+    -> stream barrier -> merge on the owner.  Total work is fixed as N grows: strong scaling."""
+    import torch
+    from paper_2608_15473_b200 import workloads as wl
+    from paper_2608_15473_b200.multi import reduce_timings, whole_job_throughput
+    from paper_2608_15473_b200.split_request import SplitPlan, cuda_runner
+
+    w = wl.config4(seed=args.seed)
+    plan = SplitPlan(world=world, rank=rank, max_shards=w.max_shards)
+    runner, out, lse, dw = cuda_runner(w, plan, dist, device, transport=args.split_transport)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        runner.step()
+    barrier()
+    assert dw.status() == 0
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(3):
+        runner.step()
+    b.record(stream)
+    barrier()
+    est = reduce_timings({"est": a.elapsed_time(b) / 3}, {}, dist, device)[0]["est"]
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+    gpu_id = vis.split(",")[local_rank].strip() if vis and local_rank < len(vis.split(",")) else str(local_rank)
+    try:
+        uuid = str(torch.cuda.get_device_properties(device).uuid)
+    except Exception:
+        uuid = None
+    with ClockSampler(gpu_id, uuid) as clocks:
+        ms, mhz, windows = time_repeats(runner.step, args.steps, n_repeats(est, args.steps), stream, barrier, clocks)
+    timing = spread(ms, mhz)
+    local_tokens = float(dw.w.swept_tokens())
+    times, counts = reduce_timings({"step": timing["median_ms"]}, {"tokens": local_tokens}, dist, device)
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        ms_per_step = times["step"]
+        total_bytes = float(w.algorithmic_bytes())
+        value = whole_job_throughput(total_bytes, ms_per_step)
+        B, Hq, D = w.batch, w.num_q_heads, w.head_dim
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": workload_name(4) + f", the cache split over {world} GPU(s)", "seed": args.seed,
+                       "shards_per_gpu": plan.per_rank, "cached_tokens_total": w.total_tokens,
+                       "l2": "inputs larger than L2 (each rank's KV slice >> 126 MB), no flush needed",
+                       "parallelism": f"one request's KV shards over {world} GPU(s); query broadcast, shard states "
+                                      f"{'stored into the owner arrays through peer-mapped memory' if args.split_transport == 'parked' else 'all-gathered'}, "
+                                      "merge on the owner",
+                       "transport": args.split_transport},
+            "timing": timing, "clocks": clocks.summary(windows),
+            "gpu_launches": 4 * args.steps,
+            "exchange": {"query_bytes_out_per_rank": B * Hq * D * 2,
+                         "state_bytes_back_per_rank": B * plan.per_rank * Hq * (D + 2) * 4,
+                         "kv_bytes_moved": 0},
+            "kv_tokens_per_s": counts["tokens"] / (ms_per_step * 1e-3),
+            "pct_of_hbm_peak": 100.0 * value / (DATASHEET_HBM_GBS * world),
+            "pct_of_measured_copy": 100.0 * value / (peak * world),
+        }
+        if not args.no_cpu_baseline:
+            from oracle import qf_oracle as orc
+            orc.build()
+            sh = orc.Shape(batch=w.batch, num_q_heads=w.num_q_heads, num_kv_heads=w.num_kv_heads,
+                           max_pages_per_req=w.max_pages_per_req, max_shards=w.max_shards)
+            t0 = time.perf_counter()
+            ref_out, ref_lse = orc.decode_full(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, sh)
+            dt = time.perf_counter() - t0
+            got_out, got_lse = out.cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+            line["parity"] = {"max_abs_out": float(np.abs(got_out - ref_out).max()),
+                              "max_rel_lse": float((np.abs(got_lse - ref_lse) / np.maximum(1.0, np.abs(ref_lse))).max()),
+                              "tolerance": {"out_max_abs": 2e-3, "lse_rel": 1e-5},
+                              "against": "the CPU oracle's unsharded sweep of the whole request"}
+            line["cpu_baseline"] = {"value": total_bytes / dt / 1e9, "unit": "GB/s", "cores": orc.num_threads(),
+                                    "kind": "oracle", "seconds": dt, "sample": "the whole request once, unsharded"}
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def run_cuda(args):
     import torch
     from paper_2608_15473_b200 import binding as qf
@@ -488,9 +578,7 @@ def run_cuda(args):
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
     if args.split_request:
-        from paper_2608_15473_b200 import split_request
-        return split_request.bench(args, dist, rank, world, device, METRIC, workload_name, ClockSampler,
-                                   measured_peaks, DATASHEET_HBM_GBS, spread, n_repeats, time_repeats)
+        return run_split_request(args, dist, rank, world, local_rank, device)
 
     # every rank owns its own batch of requests (weak scaling): seed + rank
     w = wl.CONFIGS[args.workload](seed=args.seed + rank)
@@ -640,6 +728,8 @@ def main():
     ap.add_argument("--split-request", action="store_true",
                     help="N ranks hold slices of ONE request's cache (the one-million-token workload) and write "
                          "their shard states into the owner's arrays through peer-mapped memory (strong scaling)")
+    ap.add_argument("--split-transport", default="parked", choices=["parked", "gather"],
+                    help="with --split-request: shard states stored straight into the owner's arrays (default) or all-gathered")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-also", action="store_true", help="time the headline configuration only")
     ap.add_argument("--profile-mode", action="store_true",

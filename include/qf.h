@@ -19,7 +19,8 @@
  * attention output and its log-sum-exp.  Around them: qf_combine_self and
  * qf_append_kv (the current token's fold and cache write, Section 2),
  * qf_decode_step_host (one step from host buffers), qf_project_pair (the
- * cache side's W_o / W_q projections at a layer boundary, Section 4).
+ * cache side's W_o / W_q projections at a layer boundary, Section 4),
+ * qf_enable_peer_access (a request's cache split over GPUs, Section 5).
  *
  * Readings fixed at this boundary where the paper is silent:
  *   - grouped-query attention: query head h reads KV head h / G, G = Hq/Hkv;
@@ -107,7 +108,8 @@ enum {
     QF_ERR_UNSUPPORTED = -3, /* head_dim != 128, page_size != 16, G not in 1..8     */
     QF_ERR_WORKSPACE   = -4, /* workspace NULL, misaligned (256 B) or too small    */
     QF_ERR_CUDA        = -5, /* a CUDA call failed; text via qf_strerror           */
-    QF_ERR_DEVICE      = -6, /* device is not compute capability 10.x             */
+    QF_ERR_DEVICE      = -6, /* device is not compute capability 10.x, or cannot
+                                reach the peer given to qf_enable_peer_access     */
     QF_ERR_STATIC_SCRATCH = -7 /* problem too large for qf_decode_partial_static   */
 };
 
@@ -188,6 +190,24 @@ int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache,
                       float *o_part, float *m_part, float *lse_part,
                       const qf_params *p, void *workspace, size_t workspace_bytes,
                       void *cuda_stream);
+
+/*
+ * Section 5 across devices (a request's cache split over GPUs) with Section 3's
+ * arrangement that a result is left in memory its reader can reach: before a
+ * device's qf_decode_partial may store shard states into arrays that live on
+ * another GPU (out_shards / out_shard_offset above, o_part / m_part / lse_part
+ * being pointers into the merging GPU's memory, for example CUDA IPC mappings),
+ * the CURRENT device must be allowed to access that GPU.  This call checks that
+ * it can (cudaDeviceCanAccessPeer) and enables it for the calling process
+ * (cudaDeviceEnablePeerAccess; already enabled counts as success; the same
+ * device is a no-op).  It changes no setting of a GPU that outlasts the process.
+ * Returns QF_ERR_DEVICE if the two GPUs cannot reach each other, QF_ERR_CUDA on
+ * any other failure.  Only those three output arrays may be peer memory: q, the
+ * KV pools, the tables and the workspace must be local to the GPU that runs the
+ * call (K/V tiles are fetched by TMA, which this library never points at
+ * another GPU's memory).
+ */
+int qf_enable_peer_access(int peer_device);
 
 /*
  * Section 5 merge, n-way: for every (b, h), over shards s < shard_counts[b]

@@ -42,7 +42,7 @@ EXPORTS = (
     "qf_set_profile_events", "qf_decode_partial_static", "qf_static_scratch_error",
     "qf_combine_self", "qf_append_kv", "qf_selftest_bounded_wait", "qf_plan_pieces",
     "qf_project_workspace_bytes", "qf_project_pair", "qf_project_status", "qf_fold_append",
-    "qf_static_scratch_status", "qf_project_status_inject",
+    "qf_static_scratch_status", "qf_project_status_inject", "qf_enable_peer_access",
 )
 
 
@@ -113,6 +113,8 @@ def lib() -> ctypes.CDLL:
         L.qf_static_scratch_error.restype = ctypes.c_char_p
         L.qf_static_scratch_status.restype = ctypes.c_int
         L.qf_static_scratch_status.argtypes = [ctypes.POINTER(ctypes.c_int32), vp]
+        L.qf_enable_peer_access.restype = ctypes.c_int
+        L.qf_enable_peer_access.argtypes = [ctypes.c_int]
         L.qf_project_status_inject.restype = ctypes.c_int
         L.qf_project_status_inject.argtypes = [vp, ctypes.c_int32, vp]
         L.qf_fold_append.restype = ctypes.c_int
@@ -212,6 +214,15 @@ def static_scratch_status(stream=None) -> int:
     if rc != QF_OK:
         raise QFError(rc, "qf_static_scratch_status")
     return int(st.value)
+
+
+def enable_peer_access(peer_device: int, check: bool = True) -> int:
+    """Let the current device's kernels store into memory of ``peer_device`` (shard states left in the merging
+    GPU's arrays)."""
+    rc = lib().qf_enable_peer_access(int(peer_device))
+    if check and rc != QF_OK:
+        raise QFError(rc, "qf_enable_peer_access")
+    return rc
 
 
 def project_status_inject(workspace, bits: int, stream=None) -> None:

@@ -126,7 +126,7 @@ const char *qf_strerror(int status)
     case QF_ERR_UNSUPPORTED: return "unsupported: head_dim must be 128, page_size 16, group size 1 to 8";
     case QF_ERR_WORKSPACE: return "workspace is NULL, not 256-byte aligned, or too small";
     case QF_ERR_CUDA: return g_cuda_msg[0] ? g_cuda_msg : "CUDA error";
-    case QF_ERR_DEVICE: return "device is not compute capability 10.x (this library is built for sm_100a only)";
+    case QF_ERR_DEVICE: return "device is not compute capability 10.x (this library is built for sm_100a only), or cannot reach the peer";
     case QF_ERR_STATIC_SCRATCH: return "problem needs more scratch than the built-in static array; use qf_decode_partial";
     default: return "unknown status";
     }
@@ -189,6 +189,26 @@ int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache, c
                           sizeof g_cuda_msg, &launches);
     g_last_launches = launches;
     return rc;
+}
+
+int qf_enable_peer_access(int peer_device)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (peer_device < 0) return QF_ERR_BAD_SHAPE;
+    if (peer_device == dev) return QF_OK;
+    int can = 0;
+    e = cudaDeviceCanAccessPeer(&can, dev, peer_device);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceCanAccessPeer");
+    if (!can) return QF_ERR_DEVICE;
+    e = cudaDeviceEnablePeerAccess(peer_device, 0);
+    if (e == cudaErrorPeerAccessAlreadyEnabled) {
+        cudaGetLastError();   // not an error here: clear it
+        return QF_OK;
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceEnablePeerAccess");
+    return QF_OK;
 }
 
 namespace {
