@@ -18,6 +18,7 @@
  * head); qf_combine merges a request's shard states into the full-context
  * attention output and its log-sum-exp.  Around them: qf_combine_self and
  * qf_append_kv (the current token's fold and cache write, Section 2),
+ * qf_decode_step (sweep and merge as one call, cheaper for small sweeps),
  * qf_decode_step_host (one step from host buffers), qf_project_pair (the
  * cache side's W_o / W_q projections at a layer boundary, Section 4),
  * qf_enable_peer_access (a request's cache split over GPUs, Section 5).
@@ -143,7 +144,11 @@ typedef struct qf_params {
     int32_t out_shards;        /* qf_decode_partial only: shard slots per request of
                                   the OUTPUT arrays (0 = max_shards)             */
     int32_t out_shard_offset;  /* ... and the slot this call's shard 0 goes to    */
-    int32_t reserved;          /* set to 0                                       */
+    int32_t max_seq_len;       /* 0, or an upper bound on seq_lens that the caller
+                                  guarantees (a longer length is treated as this
+                                  bound).  It lets the library recognise small
+                                  sweeps when the block-table rows are much wider
+                                  than the batch's contexts (see qf_decode_step)  */
 } qf_params;
 
 /* Library version (QF_VERSION of the build). */
@@ -190,6 +195,30 @@ int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache,
                       float *o_part, float *m_part, float *lse_part,
                       const qf_params *p, void *workspace, size_t workspace_bytes,
                       void *cuda_stream);
+
+/*
+ * Section 2, what the device returns for a step: the sweep of qf_decode_partial
+ * and the merge of qf_combine as ONE call, same arguments, same results within
+ * fp32 summation order: the shard states in o_part / m_part / lse_part and the
+ * merged out [B, Hq, D], lse [B, Hq] over shards s < shard_counts[b] (NULL = all).
+ * What the one call buys: a SMALL sweep is followed by one kernel instead of
+ * two.  When the parameters bound the work to at most 16 stage units (of 128
+ * tokens of one KV head) per SM -- batch * max_shards * num_kv_heads *
+ * ceil(T / 128) <= 16 * SMs with T = min(page_size * max_pages_per_req,
+ * max_seq_len), and max_shards <= 32 -- the pieces the sweep's schedule cut and
+ * the request's shards are merged by a single kernel that has planned its work
+ * while the sweep was still running, so that one dependent round trip to memory
+ * follows the sweep instead of three to five: such a sweep is bound by launch
+ * and dependent-load latency, not by bandwidth.  Larger problems enqueue the
+ * same three kernels as the two calls.  out_shards must be 0 here.  Errors,
+ * pointers, workspace and asynchrony as for qf_decode_partial.
+ */
+int qf_decode_step(const void *q, const void *k_cache, const void *v_cache,
+                   const int32_t *block_table, const int32_t *seq_lens,
+                   const int32_t *shard_ranges, const int32_t *shard_counts,
+                   float *o_part, float *m_part, float *lse_part, float *out, float *lse,
+                   const qf_params *p, void *workspace, size_t workspace_bytes,
+                   void *cuda_stream);
 
 /*
  * Section 5 across devices (a request's cache split over GPUs) with Section 3's

@@ -29,6 +29,13 @@ extern "C" {
 enum { QF_FLAG_DRAW_ALWAYS = 8 };
 
 /*
+ * qf_params.flags bit: qf_decode_step treats no sweep as small (see there): the
+ * finish and merge kernels run as for large problems.  Lets small parity cases
+ * reach those kernels through that call too.
+ */
+enum { QF_FLAG_NO_FUSE = 32 };
+
+/*
  * Every wait inside the kernels is bounded: when its limit runs out the kernel
  * records QF_STATUS_TIMEOUT and returns instead of hanging.  This call enqueues
  * a one-warp kernel that waits, with a limit of a few thousand polls (under a

@@ -31,6 +31,7 @@ QF_FLAG_CHECK_BOUNDS = 1
 QF_FLAG_SIMPLE_KERNEL = 2
 QF_FLAG_DRAW_ALWAYS = 8
 QF_FLAG_KV_NHD = 16
+QF_FLAG_NO_FUSE = 32
 
 QF_STATUS_BAD_PAGE = 1
 QF_STATUS_TIMEOUT = 2
@@ -42,7 +43,7 @@ EXPORTS = (
     "qf_set_profile_events", "qf_decode_partial_static", "qf_static_scratch_error",
     "qf_combine_self", "qf_append_kv", "qf_selftest_bounded_wait", "qf_plan_pieces",
     "qf_project_workspace_bytes", "qf_project_pair", "qf_project_status", "qf_fold_append",
-    "qf_static_scratch_status", "qf_project_status_inject", "qf_enable_peer_access",
+    "qf_static_scratch_status", "qf_project_status_inject", "qf_enable_peer_access", "qf_decode_step",
 )
 
 
@@ -60,7 +61,7 @@ class QFParams(ctypes.Structure):
         ("sm_scale", ctypes.c_float),
         ("out_shards", ctypes.c_int32),
         ("out_shard_offset", ctypes.c_int32),
-        ("reserved", ctypes.c_int32),
+        ("max_seq_len", ctypes.c_int32),
     ]
 
 
@@ -93,6 +94,8 @@ def lib() -> ctypes.CDLL:
         L.qf_step_scratch_bytes.argtypes = [pp]
         L.qf_decode_partial.restype = ctypes.c_int
         L.qf_decode_partial.argtypes = [vp, vp, vp, i32p, i32p, i32p, vp, vp, vp, pp, vp, ctypes.c_size_t, vp]
+        L.qf_decode_step.restype = ctypes.c_int
+        L.qf_decode_step.argtypes = [vp, vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp, vp, vp, pp, vp, ctypes.c_size_t, vp]
         L.qf_combine.restype = ctypes.c_int
         L.qf_combine.argtypes = [vp, vp, i32p, vp, vp, pp, vp]
         L.qf_decode_step_host.restype = ctypes.c_int
@@ -155,9 +158,9 @@ def _stream(stream) -> Optional[int]:
 
 def params(batch: int, num_q_heads: int, num_kv_heads: int, max_pages_per_req: int, max_shards: int,
            num_pages: int, head_dim: int = 128, page_size: int = 16, flags: int = 0,
-           sm_scale: float = 0.0, out_shards: int = 0, out_shard_offset: int = 0) -> QFParams:
+           sm_scale: float = 0.0, out_shards: int = 0, out_shard_offset: int = 0, max_seq_len: int = 0) -> QFParams:
     return QFParams(batch, num_q_heads, num_kv_heads, head_dim, page_size, max_pages_per_req, max_shards,
-                    flags, num_pages, sm_scale, out_shards, out_shard_offset, 0)
+                    flags, num_pages, sm_scale, out_shards, out_shard_offset, max_seq_len)
 
 
 def version() -> int:
@@ -204,6 +207,18 @@ def decode_partial_static(q, k_cache, v_cache, block_table, seq_lens, shard_rang
     if check and rc != QF_OK:
         detail = lib().qf_static_scratch_error().decode()
         raise QFError(rc, "qf_decode_partial_static" + (f" ({detail})" if detail else ""))
+    return rc
+
+
+def decode_step(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, shard_counts, o_part, m_part, lse_part,
+                out, lse, p: QFParams, workspace, workspace_bytes: int, stream=None, check: bool = True) -> int:
+    """Sweep and merge as one call (a small sweep is followed by one merging kernel instead of two)."""
+    rc = lib().qf_decode_step(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table), _ptr(seq_lens),
+                              _ptr(shard_ranges), _ptr(shard_counts), _ptr(o_part), _ptr(m_part), _ptr(lse_part),
+                              _ptr(out), _ptr(lse), ctypes.byref(p), _ptr(workspace), int(workspace_bytes),
+                              _stream(stream))
+    if check and rc != QF_OK:
+        raise QFError(rc, "qf_decode_step")
     return rc
 
 

@@ -14,6 +14,7 @@
 #include "qf_proj.cuh"
 #include "qf_simple.cuh"
 #include "qf_sweep.cuh"
+#include "qf_merge_small.cuh"
 
 namespace {
 
@@ -34,7 +35,7 @@ int validate(const qf_params *p)
         p->max_shards <= 0 || p->num_pages <= 0 || p->head_dim <= 0 || p->page_size <= 0)
         return QF_ERR_BAD_SHAPE;
     if (p->num_q_heads % p->num_kv_heads) return QF_ERR_BAD_SHAPE;
-    if (p->out_shards < 0 || p->out_shard_offset < 0) return QF_ERR_BAD_SHAPE;
+    if (p->out_shards < 0 || p->out_shard_offset < 0 || p->max_seq_len < 0) return QF_ERR_BAD_SHAPE;
     if (p->out_shards > 0 && (long long)p->out_shard_offset + p->max_shards > p->out_shards) return QF_ERR_BAD_SHAPE;
     if (p->out_shards == 0 && p->out_shard_offset != 0) return QF_ERR_BAD_SHAPE;
     if (p->head_dim != qf::kHeadDim || p->page_size != qf::kPageSize) return QF_ERR_UNSUPPORTED;
@@ -56,6 +57,8 @@ qf::DevParams dev_params(const qf_params *p)
     d.num_kv_heads = p->num_kv_heads;
     d.group = p->num_q_heads / p->num_kv_heads;
     d.max_pages_per_req = p->max_pages_per_req;
+    d.max_tokens = qf::max_row_tokens(p->max_pages_per_req);
+    if (p->max_seq_len > 0 && p->max_seq_len < d.max_tokens) d.max_tokens = p->max_seq_len;
     d.max_shards = p->max_shards;
     d.out_shards = p->out_shards > 0 ? p->out_shards : p->max_shards;
     d.out_shard0 = p->out_shards > 0 ? p->out_shard_offset : 0;
@@ -147,12 +150,17 @@ int qf_set_profile_events(void *start_event, void *stop_event)
     return QF_OK;
 }
 
-int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache, const int32_t *block_table,
-                      const int32_t *seq_lens, const int32_t *shard_ranges, float *o_part, float *m_part,
-                      float *lse_part, const qf_params *p, void *workspace, size_t workspace_bytes,
-                      void *cuda_stream)
+namespace {
+// The sweep, shared by qf_decode_partial (shard states only) and qf_decode_step (states and the merge).
+// `step_out` / `step_lse` non-null: the caller wants the merged result too; *merged says whether the sweep
+// kernel produced it itself (small sweeps), else the caller still has to launch the merge.
+int sweep_impl(const void *q, const void *k_cache, const void *v_cache, const int32_t *block_table,
+               const int32_t *seq_lens, const int32_t *shard_ranges, const int32_t *shard_counts, float *o_part,
+               float *m_part, float *lse_part, float *step_out, float *step_lse, bool *merged, const qf_params *p,
+               void *workspace, size_t workspace_bytes, void *cuda_stream)
 {
     g_last_launches = 0;
+    if (merged) *merged = false;
     int rc = validate(p);
     if (rc != QF_OK) return rc;
     if (!q || !k_cache || !v_cache || !seq_lens || !shard_ranges || !o_part || !m_part || !lse_part)
@@ -183,12 +191,34 @@ int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache, c
         }
     }
 
+    // A whole step over a small sweep: the sweep, then ONE kernel that merges both the pieces of cut units and
+    // the request's shards (qf_merge_small.cuh) instead of the finish kernel and the merge kernel.
+    const int n_ctas = sms < qf::kMaxSweepCtas ? sms : qf::kMaxSweepCtas;
+    const bool small = step_out && step_lse && !(p->flags & QF_FLAG_NO_FUSE) && p->out_shards == 0 &&
+                       qf::sweep_is_small(P, n_ctas);
     int launches = 0;
     rc = qf::launch_sweep(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P,
                           (char *)workspace, wsl, sms, epoch, st, g_prof_start, g_prof_stop, g_cuda_msg,
-                          sizeof g_cuda_msg, &launches);
+                          sizeof g_cuda_msg, &launches, small);
+    if (rc == QF_OK && small) {
+        cudaError_t e = qf::launch_merge_small(seq_lens, shard_ranges, shard_counts, (char *)workspace, wsl, o_part,
+                                               m_part, lse_part, step_out, step_lse, n_ctas, P, st);
+        if (e != cudaSuccess) return cuda_fail(e, "merge_small_kernel launch");
+        launches += 1;
+        if (merged) *merged = true;
+    }
     g_last_launches = launches;
     return rc;
+}
+}  // namespace
+
+int qf_decode_partial(const void *q, const void *k_cache, const void *v_cache, const int32_t *block_table,
+                      const int32_t *seq_lens, const int32_t *shard_ranges, float *o_part, float *m_part,
+                      float *lse_part, const qf_params *p, void *workspace, size_t workspace_bytes,
+                      void *cuda_stream)
+{
+    return sweep_impl(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, nullptr, o_part, m_part, lse_part,
+                      nullptr, nullptr, nullptr, p, workspace, workspace_bytes, cuda_stream);
 }
 
 int qf_enable_peer_access(int peer_device)
@@ -241,6 +271,31 @@ int qf_combine(const float *o_part, const float *lse_part, const int32_t *shard_
                const qf_params *p, void *cuda_stream)
 {
     return launch_combine(o_part, lse_part, shard_counts, nullptr, nullptr, nullptr, out, lse, p, cuda_stream);
+}
+
+int qf_decode_step(const void *q, const void *k_cache, const void *v_cache, const int32_t *block_table,
+                   const int32_t *seq_lens, const int32_t *shard_ranges, const int32_t *shard_counts,
+                   float *o_part, float *m_part, float *lse_part, float *out, float *lse, const qf_params *p,
+                   void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!out || !lse) {
+        g_last_launches = 0;
+        const int rc0 = validate(p);
+        return rc0 != QF_OK ? rc0 : QF_ERR_NULL;
+    }
+    if (p && p->out_shards != 0) {   // the step owns the merge: its shard table is the whole one
+        g_last_launches = 0;
+        const int rc0 = validate(p);
+        return rc0 != QF_OK ? rc0 : QF_ERR_BAD_SHAPE;
+    }
+    bool merged = false;
+    int rc = sweep_impl(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, shard_counts, o_part, m_part,
+                        lse_part, out, lse, &merged, p, workspace, workspace_bytes, cuda_stream);
+    if (rc != QF_OK || merged) return rc;
+    const int sweep_launches = g_last_launches;
+    rc = qf_combine(o_part, lse_part, shard_counts, out, lse, p, cuda_stream);
+    if (rc == QF_OK) g_last_launches += sweep_launches;
+    return rc;
 }
 
 int qf_combine_self(const float *o_part, const float *lse_part, const int32_t *shard_counts, const void *q,
@@ -394,18 +449,14 @@ int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_c
             if (e != cudaSuccess) return cuda_fail(e, "copy shard_counts");
         }
     }
-    rc = qf_decode_partial(base + L.q, k_cache, v_cache, block_table, (const int32_t *)(base + L.seq_lens),
-                           (const int32_t *)(base + L.shard_ranges), (float *)(base + L.o_part),
-                           (float *)(base + L.m_part), (float *)(base + L.lse_part), p, base + L.workspace,
-                           dev_scratch_bytes - L.workspace, cuda_stream);
+    rc = qf_decode_step(base + L.q, k_cache, v_cache, block_table, (const int32_t *)(base + L.seq_lens),
+                        (const int32_t *)(base + L.shard_ranges),
+                        shard_counts_host ? (const int32_t *)(base + L.shard_counts) : nullptr,
+                        (float *)(base + L.o_part), (float *)(base + L.m_part), (float *)(base + L.lse_part),
+                        mapped ? out_dev : (float *)(base + L.out), mapped ? lse_dev : (float *)(base + L.lse), p,
+                        base + L.workspace, dev_scratch_bytes - L.workspace, cuda_stream);
     if (rc != QF_OK) return rc;
-    const int sweep_launches = g_last_launches;
-    rc = qf_combine((const float *)(base + L.o_part), (const float *)(base + L.lse_part),
-                    shard_counts_host ? (const int32_t *)(base + L.shard_counts) : nullptr,
-                    mapped ? out_dev : (float *)(base + L.out), mapped ? lse_dev : (float *)(base + L.lse), p,
-                    cuda_stream);
-    if (rc != QF_OK) return rc;
-    g_last_launches += sweep_launches + extra_launches;
+    g_last_launches += extra_launches;
     if (!mapped) {
         e = cudaMemcpyAsync(out_host, base + L.out, B * Hq * D * 4, cudaMemcpyDeviceToHost, st);
         if (e != cudaSuccess) return cuda_fail(e, "copy out");

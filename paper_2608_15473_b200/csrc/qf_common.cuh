@@ -22,6 +22,7 @@ struct DevParams {
     int num_kv_heads;
     int group;               // G = Hq / Hkv
     int max_pages_per_req;
+    int max_tokens;          // no request is swept beyond this: min(16 * max_pages_per_req, the caller's bound)
     int max_shards;
     int out_shards;          // shard slots per request of the output arrays (>= out_shard0 + max_shards)
     int out_shard0;          // output slot of this call's shard 0

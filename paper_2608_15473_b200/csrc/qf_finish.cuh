@@ -23,47 +23,55 @@ constexpr int kFinThreads = kHeadDim;   // thread d owns channel d of all G head
 constexpr int kFinGroup   = 8;
 
 // Merge `count` states at slots slot0, slot0 + step, ...: running (acc, M, z) per head for channel d.
-template <int G>
-__device__ __forceinline__ void finish_merge_range(const float *__restrict__ seg, int seg_stride, int slot0, int step,
-                                                   int count, float (*s_mz)[2 * G], float *acc, float *M, float *z, int d)
+// `sync` is the barrier of the threads that take part (it returns false if the wait was abandoned, and the
+// merge stops); threads with active == false only keep the barrier count whole.
+template <int G, int kB, typename Sync>
+__device__ __forceinline__ bool finish_merge_range(const float *__restrict__ seg, int seg_stride, int slot0, int step,
+                                                   int count, float (*s_mz)[2 * G], float *acc, float *M, float *z, int d,
+                                                   bool active, Sync &&sync)
 {
-    constexpr int kB = (G == 8) ? 4 : 8;   // states whose loads are in flight together
+    // kB: states whose loads are in flight together
 #pragma unroll
     for (int o = 0; o < G; ++o) { acc[o] = 0.f; M[o] = neg_inf(); z[o] = 0.f; }
     for (int base = 0; base < count; base += kB) {
         float av[G][kB];
-#pragma unroll
-        for (int u = 0; u < kB; ++u) {
-            const bool on = base + u < count;
-            const float *sl = seg + (size_t)(slot0 + (on ? base + u : 0) * step) * seg_stride;
-#pragma unroll
-            for (int o = 0; o < G; ++o) av[o][u] = on ? ld_sync_f32(sl + o * kHeadDim + d) : 0.f;
-        }
         float mz = 0.f;
         const int u_mine = d / (2 * G), r_mine = d % (2 * G);   // (M, z) pairs of the batch: one word per thread
-        const bool mz_on = u_mine < kB && base + u_mine < count;
-        if (mz_on) mz = ld_sync_f32(seg + (size_t)(slot0 + (base + u_mine) * step) * seg_stride + G * kHeadDim + r_mine);
-        __syncthreads();                       // the previous batch's readers are done with s_mz
-        if (u_mine < kB) s_mz[u_mine][r_mine] = mz_on ? mz : (r_mine & 1 ? 0.f : neg_inf());
-        __syncthreads();
+        const bool mz_on = active && u_mine < kB && base + u_mine < count;
+        if (active) {
 #pragma unroll
-        for (int o = 0; o < G; ++o) {
-            float Mn = M[o];
+            for (int u = 0; u < kB; ++u) {
+                const bool on = base + u < count;
+                const float *sl = seg + (size_t)(slot0 + (on ? base + u : 0) * step) * seg_stride;
 #pragma unroll
-            for (int u = 0; u < kB; ++u) Mn = fmaxf(Mn, s_mz[u][2 * o]);
-            const float Ms = (Mn == neg_inf()) ? 0.f : Mn;
-            const float keep = fast_exp2(M[o] - Ms);   // 0 while nothing has been merged yet
-            z[o] *= keep;
-            acc[o] *= keep;
-#pragma unroll
-            for (int u = 0; u < kB; ++u) {   // fixed order: deterministic
-                const float ew = fast_exp2(s_mz[u][2 * o] - Ms);
-                z[o] = fmaf(s_mz[u][2 * o + 1], ew, z[o]);
-                acc[o] = fmaf(av[o][u], ew, acc[o]);
+                for (int o = 0; o < G; ++o) av[o][u] = on ? ld_sync_f32(sl + o * kHeadDim + d) : 0.f;
             }
-            M[o] = Mn;
+            if (mz_on) mz = ld_sync_f32(seg + (size_t)(slot0 + (base + u_mine) * step) * seg_stride + G * kHeadDim + r_mine);
+        }
+        if (!sync()) return false;             // the previous batch's readers are done with s_mz
+        if (active && u_mine < kB) s_mz[u_mine][r_mine] = mz_on ? mz : (r_mine & 1 ? 0.f : neg_inf());
+        if (!sync()) return false;
+        if (active) {
+#pragma unroll
+            for (int o = 0; o < G; ++o) {
+                float Mn = M[o];
+#pragma unroll
+                for (int u = 0; u < kB; ++u) Mn = fmaxf(Mn, s_mz[u][2 * o]);
+                const float Ms = (Mn == neg_inf()) ? 0.f : Mn;
+                const float keep = fast_exp2(M[o] - Ms);   // 0 while nothing has been merged yet
+                z[o] *= keep;
+                acc[o] *= keep;
+#pragma unroll
+                for (int u = 0; u < kB; ++u) {   // fixed order: deterministic
+                    const float ew = fast_exp2(s_mz[u][2 * o] - Ms);
+                    z[o] = fmaf(s_mz[u][2 * o + 1], ew, z[o]);
+                    acc[o] = fmaf(av[o][u], ew, acc[o]);
+                }
+                M[o] = Mn;
+            }
         }
     }
+    return true;
 }
 
 template <int G>
@@ -74,6 +82,7 @@ finish_kernel(const int4 *__restrict__ piece_info, const unsigned long long *__r
               float *__restrict__ o_part, float *__restrict__ m_part, float *__restrict__ lse_part, int n_units,
               DevParams P)
 {
+    constexpr int kFinBatch = (G == 8) ? 4 : 8;
     static_assert(kFinThreads >= 8 * 2 * G, "one (M, z) word per thread and batch");
     __shared__ float s_mz[8][2 * G];
     __shared__ int s_last;
@@ -108,7 +117,8 @@ finish_kernel(const int4 *__restrict__ piece_info, const unsigned long long *__r
             }
         }
     };
-    finish_merge_range<G>(seg, seg_stride, first_slot + seg0, 1, min(kFinGroup, nseg - seg0), s_mz, acc, M, z, d);
+    auto cta_sync = []() -> bool { __syncthreads(); return true; };
+    finish_merge_range<G, kFinBatch>(seg, seg_stride, first_slot + seg0, 1, min(kFinGroup, nseg - seg0), s_mz, acc, M, z, d, true, cta_sync);
     if (n_groups == 1) { write_final(); return; }
 
     // the group's partial state replaces the group's first segment (which only this CTA reads)
@@ -126,7 +136,7 @@ finish_kernel(const int4 *__restrict__ piece_info, const unsigned long long *__r
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    finish_merge_range<G>(seg, seg_stride, first_slot, kFinGroup, n_groups, s_mz, acc, M, z, d);
+    finish_merge_range<G, kFinBatch>(seg, seg_stride, first_slot, kFinGroup, n_groups, s_mz, acc, M, z, d, true, cta_sync);
     write_final();
 }
 

@@ -25,7 +25,7 @@ sweep_simple_kernel(const uint16_t *__restrict__ q, const uint16_t *__restrict__
     if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) header[kHdrLastEpoch] = epoch;
 
     int beg, end;
-    const int max_tokens = max_row_tokens(P.max_pages_per_req);
+    const int max_tokens = P.max_tokens;
     clamp_range(shard_ranges[(b * S + s) * 2], shard_ranges[(b * S + s) * 2 + 1], seq_lens[b], max_tokens, beg, end);
     if (P.check_bounds && seq_lens[b] > max_tokens && s == 0 && c == 0 && threadIdx.x == 0)
         epoch_or(header + kHdrStatus, epoch, kStatusBadPage);   // a length the block-table row cannot address

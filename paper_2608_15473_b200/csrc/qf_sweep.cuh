@@ -264,7 +264,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = P.max_shards, Hkv = P.num_kv_heads, Hq = P.num_q_heads;
     const int n_entries = P.batch * S;
-    const int max_tokens = max_row_tokens(P.max_pages_per_req);
+    const int max_tokens = P.max_tokens;
     volatile int *abort_flag = &sm.abort_flag;
 
     if (tid == 0) {
@@ -280,12 +280,10 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     grid_dependency_wait();     // nothing above touches global memory
     grid_launch_dependents();
     if (tid == kConsumerThreads) {
-        // the producer warp's first lane is idle during the plan below: it fetches the launch's epoch and
-        // makes sure the chunk counter carries it before anybody draws from it
+        // the producer warp's first lane is idle during the plan below: it fetches the launch's epoch
         const unsigned long long ep = launch_epoch(header, host_epoch);
         sm.epoch = ep;
         if (blockIdx.x == 0) header[kHdrLastEpoch] = ep;
-        epoch_counter_open(header + kHdrChunk, ep);
     }
 
     // ---- plan: prefix sum over (request, shard) entries, in shared memory when it fits
@@ -338,6 +336,9 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
     if (warp == kConsumerWarps) {
         // ============================ producer warp ============================
         const unsigned long long kv_policy = l2_evict_first_policy();
+        // the chunk counter must carry this launch's tag before this CTA draws from it (two round trips to L2 that
+        // sweeps without a drawn tail, the short ones, do not pay)
+        if (pg.n_chunks > 0 && lane == 0) epoch_counter_open(header + kHdrChunk, epoch);
         int stage = 0;
         uint32_t phase = 0;
         int issued = 0;
@@ -742,7 +743,7 @@ template <int G>
 int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void *q, const int32_t *bt,
                    const int32_t *sl, const int32_t *sr, float *o, float *m, float *l, const DevParams &P,
                    char *ws, const WorkspaceLayout &wsl, int n_ctas, unsigned long long epoch, cudaStream_t st,
-                   cudaEvent_t ev0, cudaEvent_t ev1, char *msg, size_t msg_len, int *launches)
+                   cudaEvent_t ev0, cudaEvent_t ev1, char *msg, size_t msg_len, int *launches, bool skip_finish)
 {
     unsigned long long *header = reinterpret_cast<unsigned long long *>(ws + wsl.header_off);
     int *prefix = reinterpret_cast<int *>(ws + wsl.prefix_off);
@@ -766,8 +767,7 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
     *launches = 0;
     const int *global_prefix = nullptr;
     if (n_entries > kMaxSmemEntries) {
-        plan_kernel<<<1, 1024, 0, st>>>(sl, sr, prefix, n_entries, P.max_shards, P.num_kv_heads,
-                                        max_row_tokens(P.max_pages_per_req));
+        plan_kernel<<<1, 1024, 0, st>>>(sl, sr, prefix, n_entries, P.max_shards, P.num_kv_heads, P.max_tokens);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) { snprintf(msg, msg_len, "plan_kernel launch: %s", cudaGetErrorString(e)); return -5; }
         global_prefix = prefix;
@@ -780,6 +780,7 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
     if (ev1) cudaEventRecord(ev1, st);
     if (e != cudaSuccess) { snprintf(msg, msg_len, "sweep_kernel launch: %s", cudaGetErrorString(e)); return -5; }
     *launches += 1;
+    if (skip_finish) return 0;   // the caller merges the cut units itself (small sweeps: merge_small_kernel)
     // one CTA per piece that can start inside a unit
     e = launch_pdl(finish_kernel<G>, dim3(n_ctas + kMaxDynChunks - 1), dim3(kFinThreads), 0, st,
                    (const int4 *)piece_info, (const unsigned long long *)header, kMaxSweepCtas + kMaxDynChunks,
@@ -793,21 +794,22 @@ int launch_sweep_g(const CUtensorMap &kmap, const CUtensorMap &vmap, const void 
 inline int launch_sweep(const void *q, const void *k_cache, const void *v_cache, const int32_t *bt,
                         const int32_t *sl, const int32_t *sr, float *o, float *m, float *l, const DevParams &P,
                         char *ws, const WorkspaceLayout &wsl, int sm_count, unsigned long long epoch,
-                        cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1, char *msg, size_t msg_len, int *launches)
+                        cudaStream_t st, cudaEvent_t ev0, cudaEvent_t ev1, char *msg, size_t msg_len, int *launches,
+                        bool skip_finish = false)
 {
     CUtensorMap kmap, vmap;
     if (make_pool_map(&kmap, k_cache, P.num_pages, P.num_kv_heads, kPageSize, P.kv_nhd != 0, msg, msg_len)) return -5;
     if (make_pool_map(&vmap, v_cache, P.num_pages, P.num_kv_heads, kPageSize, P.kv_nhd != 0, msg, msg_len)) return -5;
     const int n_ctas = sm_count < kMaxSweepCtas ? sm_count : kMaxSweepCtas;
     switch (P.group) {
-    case 1: return launch_sweep_g<1>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
-    case 2: return launch_sweep_g<2>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
-    case 3: return launch_sweep_g<3>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
-    case 4: return launch_sweep_g<4>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
-    case 5: return launch_sweep_g<5>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
-    case 6: return launch_sweep_g<6>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
-    case 7: return launch_sweep_g<7>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
-    default: return launch_sweep_g<8>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches);
+    case 1: return launch_sweep_g<1>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches, skip_finish);
+    case 2: return launch_sweep_g<2>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches, skip_finish);
+    case 3: return launch_sweep_g<3>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches, skip_finish);
+    case 4: return launch_sweep_g<4>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches, skip_finish);
+    case 5: return launch_sweep_g<5>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches, skip_finish);
+    case 6: return launch_sweep_g<6>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches, skip_finish);
+    case 7: return launch_sweep_g<7>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches, skip_finish);
+    default: return launch_sweep_g<8>(kmap, vmap, q, bt, sl, sr, o, m, l, P, ws, wsl, n_ctas, epoch, st, ev0, ev1, msg, msg_len, launches, skip_finish);
     }
 }
 

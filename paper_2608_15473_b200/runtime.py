@@ -75,7 +75,16 @@ class DeviceWorkload:
         qf.combine(self.o_part, self.lse_part, self.shard_counts, self.out, self.lse, self.params, stream)
 
     def step(self, stream=None) -> int:
-        """One pass of the whole hot path; returns the number of kernels enqueued."""
+        """One pass of the whole hot path (qf_decode_step: shard states and the merged result; the sweep, the merge
+        of cut units and the merge of shards, the last two as one kernel when the sweep is small); returns the number
+        of kernels enqueued."""
+        qf.decode_step(self.q, self.k_cache, self.v_cache, self.block_table, self.seq_lens, self.shard_ranges,
+                       self.shard_counts, self.o_part, self.m_part, self.lse_part, self.out, self.lse, self.params,
+                       self.workspace, self.ws_bytes, stream)
+        return qf.last_launch_count()
+
+    def step_two_calls(self, stream=None) -> int:
+        """The same pass as two calls, qf_decode_partial then qf_combine."""
         self.sweep(stream)
         n = qf.last_launch_count()
         self.merge(stream)

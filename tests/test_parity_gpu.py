@@ -22,10 +22,13 @@ def built():
     assert qf.version() == 100
 
 
-def run(w, flags=0, null_table=False):
+def run(w, flags=0, null_table=False, two_calls=False):
     dw = DeviceWorkload(w, flags=flags, identity_table_as_null=null_table)
     dw.poison_outputs()
-    dw.step()
+    if two_calls:
+        dw.step_two_calls()
+    else:
+        dw.step()
     return dw
 
 
@@ -37,7 +40,10 @@ KERNELS = [pytest.param((0, 16), id="unit16"), pytest.param((0, 8), id="unit8"),
            # token-major pages (the device copy is rearranged by DeviceWorkload; the oracle sees the same values)
            pytest.param((qf.QF_FLAG_KV_NHD, 8), id="nhd8"), pytest.param((qf.QF_FLAG_KV_NHD, 2), id="nhd2"),
            pytest.param((qf.QF_FLAG_KV_NHD | qf.QF_FLAG_SIMPLE_KERNEL, 2), id="simple-nhd"),
-           pytest.param((qf.QF_FLAG_KV_NHD | qf.QF_FLAG_DRAW_ALWAYS, 8), id="draw8-nhd")]
+           pytest.param((qf.QF_FLAG_KV_NHD | qf.QF_FLAG_DRAW_ALWAYS, 8), id="draw8-nhd"),
+           # a whole step over a small sweep merges with one kernel by default; these keep the finish and merge kernels
+           pytest.param((qf.QF_FLAG_NO_FUSE, 8), id="nofuse8"), pytest.param((qf.QF_FLAG_NO_FUSE, 2), id="nofuse2"),
+           pytest.param((qf.QF_FLAG_NO_FUSE | qf.QF_FLAG_DRAW_ALWAYS, 8), id="nofuse-draw8")]
 
 
 # T1: every short length, both group sizes, shuffled table: tail-page masking, first-tile guard
@@ -569,3 +575,63 @@ def test_split_request_written_in_place_by_virtual_ranks(world, flags):
         assert T.out_err(got_o[:, dst], ref_o[:, sl.start:sl.stop]) <= T.ENG_OUT
         assert T.lse_err(got_l[:, dst], ref_l[:, sl.start:sl.stop]) <= T.ENG_LSE
         assert np.isneginf(got_l[:, rank * per + len(sl):(rank + 1) * per]).all()
+
+
+# A whole step over a SMALL sweep (qf_decode_step): the pieces of cut units and the request's shards are merged by
+# one kernel that plans while the sweep runs.  Against the oracle, against the three-kernel path, and bit for bit
+# against itself over repeated launches.
+@pytest.mark.parametrize("Hkv,G", [(8, 2), (8, 4), (2, 8), (1, 1), (4, 7), (16, 2), (8, 5)])
+def test_small_sweeps_merge_with_one_kernel(Hkv, G):
+    rng = np.random.default_rng(Hkv * 10 + G)
+    cases = [
+        ([4096], [[(0, 4096)]]),                                     # one request, one shard: every unit cut ~16 times
+        ([3000, 0, 17, 1200], [wl.even_shards(L, 3) for L in (3000, 0, 17, 1200)]),
+        ([900] * 6, [[(0, 100), (100, 100), (100, 900), (950, 2000)]] * 6),   # empty and out-of-range shards
+        ([int(x) for x in rng.integers(1, 2000, size=9)], None),
+        ([5000, 64], [wl.even_shards(L, 20) for L in (5000, 64)]),   # more uncut shards than one batch holds
+    ]
+    for lens, ranges in cases:
+        if ranges is None:
+            ranges = [wl.fixed_shards(L, 512) for L in lens]
+        w = wl.make_workload("small", lens, ranges, Hkv * G, Hkv, seed=G + len(lens), poison_tails=True,
+                             pool_factor=1.25, poison_unused=True)
+        dw = run(w)
+        small = w.batch * w.max_shards * Hkv * (-(-w.max_pages_per_req // 8)) <= 16 * 148 and w.max_shards <= 32
+        assert qf.last_launch_count() == (2 if small else 3)
+        T.compare_all(dw, w, tag=f"Hkv={Hkv} G={G} lens={lens[:4]}")
+        assert dw.status() == 0
+        first = [r.copy() for r in dw.results()]
+        for _ in range(3):
+            dw.poison_outputs()
+            dw.step()
+            for x, y in zip(first, dw.results()):
+                assert np.array_equal(x, y)
+        # the same as two calls, and as one call with the small path switched off: three kernels, same results
+        # within fp32 summation order
+        for dw3 in (run(w, two_calls=True), run(w, qf.QF_FLAG_NO_FUSE)):
+            assert qf.last_launch_count() in (1, 3)      # the merge alone, or sweep + finish + merge
+            T.compare_all(dw3, w)
+            for x, y in zip(dw.results(), dw3.results()):
+                assert np.allclose(x, y, rtol=0, atol=T.ENG_OUT, equal_nan=True)
+
+
+def test_small_sweep_honours_shard_counts_and_the_length_bound():
+    # shards past shard_counts[b] are swept but not merged; a max_seq_len bound makes a wide table small
+    lens = [700, 300, 64]
+    ranges = [[(0, 200), (200, 500), (500, 700)], [(0, 300), (0, 150), (150, 300)], [(0, 64), (0, 0), (0, 64)]]
+    w = wl.make_workload("fuse-counts", lens, ranges, 8, 2, seed=3, shard_counts=[3, 1, 1], max_pages_per_req=4000)
+    dw = run(w)
+    assert qf.last_launch_count() == 3            # the table rows are wide: nothing says the sweep is small
+    T.compare_all(dw, w)
+    dw.params.max_seq_len = 1024
+    dw.poison_outputs()
+    dw.step()
+    assert qf.last_launch_count() == 2
+    T.compare_all(dw, w)
+    # a bound below a request's real length clamps it, like a short table row
+    dw.params.max_seq_len = 256
+    dw.poison_outputs()
+    dw.step()
+    w2 = wl.make_workload("fuse-counts", lens, ranges, 8, 2, seed=3, shard_counts=[3, 1, 1], max_pages_per_req=4000)
+    w2.seq_lens = np.minimum(w2.seq_lens, 256).astype(np.int32)
+    T.compare_all(dw, w2)
