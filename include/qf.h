@@ -19,7 +19,8 @@
  * attention output and its log-sum-exp.  Around them: qf_combine_self and
  * qf_append_kv (the current token's fold and cache write, Section 2),
  * qf_decode_step (sweep and merge as one call, cheaper for small sweeps),
- * qf_decode_step_host (one step from host buffers), qf_project_pair (the
+ * qf_decode_step_host (one step from host buffers; qf_host_pipe_* the same,
+ * pipelined), qf_project_pair (the
  * cache side's W_o / W_q projections at a layer boundary, Section 4),
  * qf_enable_peer_access (a request's cache split over GPUs, Section 5).
  *
@@ -364,6 +365,36 @@ int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_c
                         float *out_host, float *lse_host,
                         const qf_params *p, void *dev_scratch, size_t dev_scratch_bytes,
                         void *cuda_stream);
+
+/*
+ * The same step from host buffers, PIPELINED (Section 2: three small messages per
+ * step, and only the query has to arrive before the sweep): a queue of `depth`
+ * steps in flight.  qf_host_pipe_submit enqueues one step and returns at once
+ * with a ticket (>= 0; negative = error code): the query and the metadata travel
+ * to the device on a transfer stream of the pipe's own while earlier steps'
+ * sweeps run on `cuda_stream`, the sweep and merge follow on `cuda_stream`, and
+ * the result travels back on a second transfer stream while the next sweep runs.
+ * qf_host_pipe_wait blocks until that ticket's out_host / lse_host are complete.
+ * The caller keeps every host buffer of a step untouched from submit until its
+ * wait has returned (so it rotates `depth` sets of them), and should pass
+ * page-locked buffers: pageable ones make the copies synchronous.  Submitting
+ * when `depth` steps are in flight first waits for the oldest.
+ *   dev_scratch: qf_host_pipe_scratch_bytes(p, depth) bytes of device memory,
+ *   256-byte aligned, borrowed until destroy.  depth is 1 to 8.
+ * The pipe owns two CUDA streams and 3 * depth events (host-side objects; no
+ * device memory is allocated).  One host thread uses a pipe at a time.
+ */
+typedef struct qf_host_pipe qf_host_pipe;
+size_t qf_host_pipe_scratch_bytes(const qf_params *p, int depth);
+int qf_host_pipe_create(qf_host_pipe **pipe, const qf_params *p, void *dev_scratch,
+                        size_t dev_scratch_bytes, int depth);
+long long qf_host_pipe_submit(qf_host_pipe *pipe, const void *q_host, const void *k_cache,
+                              const void *v_cache, const int32_t *block_table,
+                              const int32_t *seq_lens_host, const int32_t *shard_ranges_host,
+                              const int32_t *shard_counts_host, float *out_host, float *lse_host,
+                              void *cuda_stream);
+int qf_host_pipe_wait(qf_host_pipe *pipe, long long ticket);
+int qf_host_pipe_destroy(qf_host_pipe *pipe);
 
 /*
  * Copies the workspace status word (QF_STATUS_* bits, 0 = clean) of the last

@@ -44,6 +44,8 @@ EXPORTS = (
     "qf_combine_self", "qf_append_kv", "qf_selftest_bounded_wait", "qf_plan_pieces",
     "qf_project_workspace_bytes", "qf_project_pair", "qf_project_status", "qf_fold_append",
     "qf_static_scratch_status", "qf_project_status_inject", "qf_enable_peer_access", "qf_decode_step",
+    "qf_host_pipe_scratch_bytes", "qf_host_pipe_create", "qf_host_pipe_submit", "qf_host_pipe_wait",
+    "qf_host_pipe_destroy",
 )
 
 
@@ -116,6 +118,16 @@ def lib() -> ctypes.CDLL:
         L.qf_static_scratch_error.restype = ctypes.c_char_p
         L.qf_static_scratch_status.restype = ctypes.c_int
         L.qf_static_scratch_status.argtypes = [ctypes.POINTER(ctypes.c_int32), vp]
+        L.qf_host_pipe_scratch_bytes.restype = ctypes.c_size_t
+        L.qf_host_pipe_scratch_bytes.argtypes = [pp, ctypes.c_int]
+        L.qf_host_pipe_create.restype = ctypes.c_int
+        L.qf_host_pipe_create.argtypes = [ctypes.POINTER(ctypes.c_void_p), pp, vp, ctypes.c_size_t, ctypes.c_int]
+        L.qf_host_pipe_submit.restype = ctypes.c_longlong
+        L.qf_host_pipe_submit.argtypes = [vp, vp, vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp]
+        L.qf_host_pipe_wait.restype = ctypes.c_int
+        L.qf_host_pipe_wait.argtypes = [vp, ctypes.c_longlong]
+        L.qf_host_pipe_destroy.restype = ctypes.c_int
+        L.qf_host_pipe_destroy.argtypes = [vp]
         L.qf_enable_peer_access.restype = ctypes.c_int
         L.qf_enable_peer_access.argtypes = [ctypes.c_int]
         L.qf_project_status_inject.restype = ctypes.c_int
@@ -296,6 +308,40 @@ def decode_step_host(q_host, k_cache, v_cache, block_table, seq_lens_host, shard
     if check and rc != QF_OK:
         raise QFError(rc, "qf_decode_step_host")
     return rc
+
+
+def host_pipe_scratch_bytes(p: QFParams, depth: int) -> int:
+    return int(lib().qf_host_pipe_scratch_bytes(ctypes.byref(p), int(depth)))
+
+
+def host_pipe_create(p: QFParams, dev_scratch, dev_scratch_bytes: int, depth: int) -> int:
+    """A pipelined host-buffer stepper; returns its handle (an integer address)."""
+    h = ctypes.c_void_p(None)
+    rc = lib().qf_host_pipe_create(ctypes.byref(h), ctypes.byref(p), _ptr(dev_scratch), int(dev_scratch_bytes), int(depth))
+    if rc != QF_OK:
+        raise QFError(rc, "qf_host_pipe_create")
+    return int(h.value)
+
+
+def host_pipe_submit(pipe: int, q_host, k_cache, v_cache, block_table, seq_lens_host, shard_ranges_host,
+                     shard_counts_host, out_host, lse_host, stream=None) -> int:
+    """Enqueue one step; returns its ticket."""
+    t = lib().qf_host_pipe_submit(pipe, _ptr(q_host), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
+                                  _ptr(seq_lens_host), _ptr(shard_ranges_host), _ptr(shard_counts_host),
+                                  _ptr(out_host), _ptr(lse_host), _stream(stream))
+    if t < 0:
+        raise QFError(int(t), "qf_host_pipe_submit")
+    return int(t)
+
+
+def host_pipe_wait(pipe: int, ticket: int) -> None:
+    rc = lib().qf_host_pipe_wait(pipe, int(ticket))
+    if rc != QF_OK:
+        raise QFError(rc, "qf_host_pipe_wait")
+
+
+def host_pipe_destroy(pipe: int) -> None:
+    lib().qf_host_pipe_destroy(pipe)
 
 
 def selftest_bounded_wait(workspace, stream=None) -> None:

@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <new>
 
 #include "../../include/qf.h"
 #include "../../include/qf_testing.h"
@@ -465,6 +466,136 @@ int qf_decode_step_host(const void *q_host, const void *k_cache, const void *v_c
     }
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    return QF_OK;
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// Steps from host buffers, pipelined: step n + 1's inputs travel in and step n's result travels out while a
+// sweep runs.  Slots of step scratch, two private transfer streams (in, out) and three events per slot.
+struct qf_host_pipe {
+    qf_params p;
+    char *scratch;
+    size_t slot_bytes;
+    int depth;
+    int device;
+    cudaStream_t s_in, s_out;
+    cudaEvent_t ev_in[8], ev_comp[8], ev_done[8];
+    long long submitted;          // tickets handed out so far
+    int launches_per_step;
+};
+
+size_t qf_host_pipe_scratch_bytes(const qf_params *p, int depth)
+{
+    if (validate(p) != QF_OK || depth < 1 || depth > 8) return 0;
+    return step_layout(p).total * (size_t)depth;
+}
+
+int qf_host_pipe_create(qf_host_pipe **pipe, const qf_params *p, void *dev_scratch, size_t dev_scratch_bytes, int depth)
+{
+    if (!pipe) return QF_ERR_NULL;
+    *pipe = nullptr;
+    int rc = validate(p);
+    if (rc != QF_OK) return rc;
+    if (depth < 1 || depth > 8 || p->out_shards != 0) return QF_ERR_BAD_SHAPE;
+    const size_t slot = step_layout(p).total;
+    if (!dev_scratch || ((uintptr_t)dev_scratch & 255) || dev_scratch_bytes < slot * (size_t)depth) return QF_ERR_WORKSPACE;
+    rc = check_device(nullptr);
+    if (rc != QF_OK) return rc;
+    qf_host_pipe *h = new (std::nothrow) qf_host_pipe();
+    if (!h) return QF_ERR_CUDA;
+    h->p = *p;
+    h->scratch = (char *)dev_scratch;
+    h->slot_bytes = slot;
+    h->depth = depth;
+    h->submitted = 0;
+    h->launches_per_step = 0;
+    cudaGetDevice(&h->device);
+    cudaError_t e = cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking);
+    for (int i = 0; i < depth && e == cudaSuccess; ++i) {
+        e = cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_comp[i], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming);
+    }
+    if (e != cudaSuccess) {
+        delete h;     // streams and events made so far are released with the context; creation does not fail in practice
+        return cuda_fail(e, "qf_host_pipe_create");
+    }
+    *pipe = h;
+    return QF_OK;
+}
+
+long long qf_host_pipe_submit(qf_host_pipe *h, const void *q_host, const void *k_cache, const void *v_cache,
+                              const int32_t *block_table, const int32_t *seq_lens_host,
+                              const int32_t *shard_ranges_host, const int32_t *shard_counts_host, float *out_host,
+                              float *lse_host, void *cuda_stream)
+{
+    if (!h || !q_host || !k_cache || !v_cache || !seq_lens_host || !shard_ranges_host || !out_host || !lse_host)
+        return QF_ERR_NULL;
+    const qf_params *p = &h->p;
+    const long long ticket = h->submitted;
+    const int slot = (int)(ticket % h->depth);
+    cudaError_t e;
+    if (ticket >= h->depth) {   // the slot's previous step must have left it
+        e = cudaEventSynchronize(h->ev_done[slot]);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventSynchronize");
+    }
+    const StepLayout L = step_layout(p);
+    char *base = h->scratch + (size_t)slot * h->slot_bytes;
+    const size_t B = p->batch, S = p->max_shards, Hq = p->num_q_heads, D = p->head_dim;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // in: the query and the step's metadata, on the inbound stream
+    e = cudaMemcpyAsync(base + L.q, q_host, B * Hq * D * 2, cudaMemcpyHostToDevice, h->s_in);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(base + L.seq_lens, seq_lens_host, B * 4, cudaMemcpyHostToDevice, h->s_in);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(base + L.shard_ranges, shard_ranges_host, B * S * 8, cudaMemcpyHostToDevice, h->s_in);
+    if (e == cudaSuccess && shard_counts_host)
+        e = cudaMemcpyAsync(base + L.shard_counts, shard_counts_host, B * 4, cudaMemcpyHostToDevice, h->s_in);
+    if (e == cudaSuccess) e = cudaEventRecord(h->ev_in[slot], h->s_in);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, h->ev_in[slot], 0);
+    if (e != cudaSuccess) return cuda_fail(e, "qf_host_pipe_submit (inbound)");
+    // the step itself, on the caller's stream
+    const int rc = qf_decode_step(base + L.q, k_cache, v_cache, block_table, (const int32_t *)(base + L.seq_lens),
+                                  (const int32_t *)(base + L.shard_ranges),
+                                  shard_counts_host ? (const int32_t *)(base + L.shard_counts) : nullptr,
+                                  (float *)(base + L.o_part), (float *)(base + L.m_part), (float *)(base + L.lse_part),
+                                  (float *)(base + L.out), (float *)(base + L.lse), p, base + L.workspace,
+                                  h->slot_bytes - L.workspace, cuda_stream);
+    if (rc != QF_OK) return rc;
+    h->launches_per_step = g_last_launches;
+    // out: the result, on the outbound stream
+    e = cudaEventRecord(h->ev_comp[slot], st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->s_out, h->ev_comp[slot], 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out_host, base + L.out, B * Hq * D * 4, cudaMemcpyDeviceToHost, h->s_out);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(lse_host, base + L.lse, B * Hq * 4, cudaMemcpyDeviceToHost, h->s_out);
+    if (e == cudaSuccess) e = cudaEventRecord(h->ev_done[slot], h->s_out);
+    if (e != cudaSuccess) return cuda_fail(e, "qf_host_pipe_submit (outbound)");
+    h->submitted = ticket + 1;
+    return ticket;
+}
+
+int qf_host_pipe_wait(qf_host_pipe *h, long long ticket)
+{
+    if (!h) return QF_ERR_NULL;
+    if (ticket < 0 || ticket >= h->submitted) return QF_ERR_BAD_SHAPE;
+    if (ticket + h->depth < h->submitted) return QF_OK;   // its slot has been reused: that step was waited for then
+    const cudaError_t e = cudaEventSynchronize(h->ev_done[(int)(ticket % h->depth)]);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaEventSynchronize");
+    return QF_OK;
+}
+
+int qf_host_pipe_destroy(qf_host_pipe *h)
+{
+    if (!h) return QF_OK;
+    cudaStreamSynchronize(h->s_in);
+    cudaStreamSynchronize(h->s_out);
+    for (int i = 0; i < h->depth; ++i) {
+        cudaEventDestroy(h->ev_in[i]);
+        cudaEventDestroy(h->ev_comp[i]);
+        cudaEventDestroy(h->ev_done[i]);
+    }
+    cudaStreamDestroy(h->s_in);
+    cudaStreamDestroy(h->s_out);
+    delete h;
     return QF_OK;
 }
 

@@ -136,6 +136,63 @@ class HostStepper:
             raise qf.QFError(rc, "qf_decode_step_host")
 
 
+class HostPipeline:
+    """Steps from pinned host buffers with ``depth`` steps in flight (qf_host_pipe_*): a step's query travels in and
+    the previous step's result travels out while a sweep runs.  Holds ``depth`` rotating sets of host buffers;
+    ``submit`` takes the step's query (bf16 bit patterns, any integer-16 tensor or array of the right size) and
+    returns a ticket, ``wait`` returns that step's (out, lse) host tensors, valid until the slot is reused."""
+
+    def __init__(self, dw: DeviceWorkload, depth: int = 2):
+        self.dw, self.depth = dw, depth
+        w = dw.w
+        pin = lambda t: t.pin_memory()
+        self.q_host = [pin(torch.from_numpy(w.q.view(np.int16).copy())) for _ in range(depth)]
+        self.seq_lens_host = [pin(torch.from_numpy(w.seq_lens.copy())) for _ in range(depth)]
+        self.shard_ranges_host = [pin(torch.from_numpy(w.shard_ranges.copy())) for _ in range(depth)]
+        self.shard_counts_host = [pin(torch.from_numpy(w.shard_counts.copy())) for _ in range(depth)]
+        self.out_host = [pin(torch.empty((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32)) for _ in range(depth)]
+        self.lse_host = [pin(torch.empty((w.batch, w.num_q_heads), dtype=torch.float32)) for _ in range(depth)]
+        self.scratch_bytes = qf.host_pipe_scratch_bytes(dw.params, depth)
+        self.scratch = torch.empty(self.scratch_bytes, dtype=torch.uint8, device=dw.device)
+        self.pipe = qf.host_pipe_create(dw.params, self.scratch, self.scratch_bytes, depth)
+        self.h2d_bytes = (self.q_host[0].numel() * 2 + self.seq_lens_host[0].numel() * 4 +
+                          self.shard_ranges_host[0].numel() * 4 + self.shard_counts_host[0].numel() * 4)
+        self.d2h_bytes = self.out_host[0].numel() * 4 + self.lse_host[0].numel() * 4
+        self._next = 0
+
+    def submit(self, q_bits=None, stream=None) -> int:
+        """Enqueue one step (with a new query if given: written into the slot's pinned buffer first)."""
+        slot = self._next % self.depth
+        if self._next >= self.depth:
+            qf.host_pipe_wait(self.pipe, self._next - self.depth)     # the slot's host buffers are free again
+        if q_bits is not None:
+            src = torch.as_tensor(np.ascontiguousarray(q_bits).view(np.int16)) if not torch.is_tensor(q_bits) else q_bits
+            self.q_host[slot].copy_(src.view(torch.int16).reshape(self.q_host[slot].shape))
+        dw = self.dw
+        t = qf.host_pipe_submit(self.pipe, self.q_host[slot], dw.k_cache, dw.v_cache, dw.block_table,
+                                self.seq_lens_host[slot], self.shard_ranges_host[slot], self.shard_counts_host[slot],
+                                self.out_host[slot], self.lse_host[slot], stream)
+        assert t == self._next
+        self._next += 1
+        return t
+
+    def wait(self, ticket: int):
+        qf.host_pipe_wait(self.pipe, ticket)
+        slot = ticket % self.depth
+        return self.out_host[slot], self.lse_host[slot]
+
+    def close(self) -> None:
+        if self.pipe:
+            qf.host_pipe_destroy(self.pipe)
+            self.pipe = 0
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
 class CacheSideStack:
     """The cache side of a stack of layers for one batch of co-resident requests (Section 4): per layer its KV
     pool, W_o, W_q and the normalisation gain.  A stage of layer l is what the cache side does per token and layer:

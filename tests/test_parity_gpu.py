@@ -9,7 +9,7 @@ from oracle import qf_oracle as orc
 from paper_2608_15473_b200 import binding as qf
 from paper_2608_15473_b200 import build as qf_build
 from paper_2608_15473_b200 import workloads as wl
-from paper_2608_15473_b200.runtime import DeviceWorkload, HostStepper
+from paper_2608_15473_b200.runtime import DeviceWorkload, HostPipeline, HostStepper
 
 import qf_testlib as T
 
@@ -635,3 +635,40 @@ def test_small_sweep_honours_shard_counts_and_the_length_bound():
     w2 = wl.make_workload("fuse-counts", lens, ranges, 8, 2, seed=3, shard_counts=[3, 1, 1], max_pages_per_req=4000)
     w2.seq_lens = np.minimum(w2.seq_lens, 256).astype(np.int32)
     T.compare_all(dw, w2)
+
+
+@pytest.mark.parametrize("depth", [1, 2, 3])
+def test_pipelined_host_steps_match_the_device_path(depth):
+    # steps in flight with different queries: every ticket's result equals the device-resident step on that query,
+    # bit for bit, whatever overlaps with whatever; host buffers rotate with the pipe's slots
+    w = wl.config3(seed=11, batch=5, hi=7000)
+    dw = DeviceWorkload(w)
+    pipe = HostPipeline(dw, depth=depth)
+    rng = np.random.default_rng(depth)
+    queries = [wl.f32_to_bf16_bits(rng.standard_normal(w.q.shape).astype(np.float32)) for _ in range(7)]
+    want = []
+    for qb in queries:
+        dw.q.copy_(torch.from_numpy(qb.view(np.int16)).view(torch.bfloat16).cuda())
+        dw.poison_outputs()
+        dw.step()
+        _, _, _, out, lse = dw.results()
+        want.append((out, lse))
+    tickets = []
+    got = {}
+    for i, qb in enumerate(queries):
+        tickets.append(pipe.submit(qb))
+        if i >= depth - 1:                      # keep `depth` steps in flight, collect the oldest
+            t = tickets[i - (depth - 1)]
+            out, lse = pipe.wait(t)
+            got[t] = (out.numpy().astype(np.float64).copy(), lse.numpy().astype(np.float64).copy())
+    for t in tickets:
+        if t not in got:
+            out, lse = pipe.wait(t)
+            got[t] = (out.numpy().astype(np.float64).copy(), lse.numpy().astype(np.float64).copy())
+    for t, (out, lse) in zip(tickets, want):
+        assert np.array_equal(got[t][0], out) and np.array_equal(got[t][1], lse), t
+    # against the oracle for the last query
+    w.q = queries[-1]
+    ref = T.oracle_all(w)
+    assert T.out_err(got[tickets[-1]][0], ref[3]) <= T.ENG_OUT and T.lse_err(got[tickets[-1]][1], ref[4]) <= T.ENG_LSE
+    pipe.close()
