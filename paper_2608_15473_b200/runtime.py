@@ -230,9 +230,10 @@ class CacheSideStack:
         n = qf.last_launch_count()
         qf.fold_append(dw.o_part, dw.lse_part, dw.shard_counts, dw.q, k_new, v_new, dw.out, dw.lse, dw.k_cache,
                        dw.v_cache, dw.block_table, dw.seq_lens, dw.params, advance_lengths=True, stream=stream)
+        n += qf.last_launch_count()
         qf.project_pair(dw.out.view(self.batch, self.n_q), z, self.w_o[l], self.gain[l], self.w_q[l], u_out,
                         nxt.q.view(self.batch, self.n_q), self.eps, self.proj_ws, stream)
-        return n + 3
+        return n + qf.last_launch_count()
 
     def token(self, z, k_new, v_new, u_out, stream=None) -> int:
         """One token through every layer: z, k_new, v_new, u_out are [L, ...] stacks, one slice per layer."""
