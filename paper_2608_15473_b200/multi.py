@@ -19,8 +19,10 @@ def reduce_timings(times_ms: Dict[str, float], counts: Dict[str, float], dist=No
     keys_t, keys_c = sorted(times_ms), sorted(counts)
     t = torch.tensor([times_ms[k] for k in keys_t], dtype=torch.float64, device=device)
     c = torch.tensor([counts[k] for k in keys_c], dtype=torch.float64, device=device)
-    dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    if keys_t:       # an empty dictionary is not reduced at all (no zero-element collective)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    if keys_c:
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
     return ({k: float(v) for k, v in zip(keys_t, t.tolist())},
             {k: float(v) for k, v in zip(keys_c, c.tolist())})
 

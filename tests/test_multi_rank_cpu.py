@@ -30,6 +30,9 @@ def _rank_main(rank, world, port, out_dir):
         times, counts = reduce_timings({"elapsed": 10.0 + 5.0 * rank, "e2e": 30.0 - rank},
                                        {"bytes": float(w.algorithmic_bytes()), "tokens": float(w.swept_tokens())},
                                        dist, "cpu")
+        # the bench's estimate reduction: times only, no counts (nothing to sum: no collective for it)
+        est, none = reduce_timings({"est": 1.0 + rank}, {}, dist, "cpu")
+        assert est == {"est": float(world)} and none == {}
         np.save(os.path.join(out_dir, f"r{rank}.npy"),
                 np.array([times["elapsed"], times["e2e"], counts["bytes"], counts["tokens"],
                           float(w.algorithmic_bytes()), float(w.swept_tokens()), own.start, own.stop]))
