@@ -33,7 +33,7 @@ enum { QF_FLAG_DRAW_ALWAYS = 8 };
  * finish and merge kernels run as for large problems.  Lets small parity cases
  * reach those kernels through that call too.
  */
-enum { QF_FLAG_NO_FUSE = 32 };
+enum { QF_FLAG_NO_SMALL_MERGE = 32 };
 
 /*
  * Every wait inside the kernels is bounded: when its limit runs out the kernel

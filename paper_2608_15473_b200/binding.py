@@ -31,7 +31,7 @@ QF_FLAG_CHECK_BOUNDS = 1
 QF_FLAG_SIMPLE_KERNEL = 2
 QF_FLAG_DRAW_ALWAYS = 8
 QF_FLAG_KV_NHD = 16
-QF_FLAG_NO_FUSE = 32
+QF_FLAG_NO_SMALL_MERGE = 32
 
 QF_STATUS_BAD_PAGE = 1
 QF_STATUS_TIMEOUT = 2

@@ -195,7 +195,7 @@ int sweep_impl(const void *q, const void *k_cache, const void *v_cache, const in
     // A whole step over a small sweep: the sweep, then ONE kernel that merges both the pieces of cut units and
     // the request's shards (qf_merge_small.cuh) instead of the finish kernel and the merge kernel.
     const int n_ctas = sms < qf::kMaxSweepCtas ? sms : qf::kMaxSweepCtas;
-    const bool small = step_out && step_lse && !(p->flags & QF_FLAG_NO_FUSE) && p->out_shards == 0 &&
+    const bool small = step_out && step_lse && !(p->flags & QF_FLAG_NO_SMALL_MERGE) && p->out_shards == 0 &&
                        qf::sweep_is_small(P, n_ctas);
     int launches = 0;
     rc = qf::launch_sweep(q, k_cache, v_cache, block_table, seq_lens, shard_ranges, o_part, m_part, lse_part, P,
@@ -518,7 +518,7 @@ int qf_host_pipe_create(qf_host_pipe **pipe, const qf_params *p, void *dev_scrat
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming);
     }
     if (e != cudaSuccess) {
-        delete h;     // streams and events made so far are released with the context; creation does not fail in practice
+        qf_host_pipe_destroy(h);   // releases whatever was created (the rest of the handles are null)
         return cuda_fail(e, "qf_host_pipe_create");
     }
     *pipe = h;
@@ -586,15 +586,15 @@ int qf_host_pipe_wait(qf_host_pipe *h, long long ticket)
 int qf_host_pipe_destroy(qf_host_pipe *h)
 {
     if (!h) return QF_OK;
-    cudaStreamSynchronize(h->s_in);
-    cudaStreamSynchronize(h->s_out);
+    if (h->s_in) cudaStreamSynchronize(h->s_in);
+    if (h->s_out) cudaStreamSynchronize(h->s_out);
     for (int i = 0; i < h->depth; ++i) {
-        cudaEventDestroy(h->ev_in[i]);
-        cudaEventDestroy(h->ev_comp[i]);
-        cudaEventDestroy(h->ev_done[i]);
+        if (h->ev_in[i]) cudaEventDestroy(h->ev_in[i]);
+        if (h->ev_comp[i]) cudaEventDestroy(h->ev_comp[i]);
+        if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
     }
-    cudaStreamDestroy(h->s_in);
-    cudaStreamDestroy(h->s_out);
+    if (h->s_in) cudaStreamDestroy(h->s_in);
+    if (h->s_out) cudaStreamDestroy(h->s_out);
     delete h;
     return QF_OK;
 }

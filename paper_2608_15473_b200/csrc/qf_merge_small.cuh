@@ -1,6 +1,6 @@
 // The merge of a SMALL sweep in one kernel: the pieces of the (shard, KV head) units that the sweep's schedule
 // cut, and then the request's shards (Section 5: states of disjoint sets add, in any order), for a sweep that
-// qf_decode_step knows to be small (at most kFuseUnitsPerCta stage units per CTA by a bound the host can compute).
+// qf_decode_step knows to be small (at most kSmallUnitsPerCta stage units per CTA by a bound the host can compute).
 //
 // A small sweep is bound by launch and dependent-load latency, not by bandwidth, and what follows it decides its
 // latency: the general path runs the finish kernel (piece record, then segments; a second level for units of more
@@ -27,7 +27,7 @@
 
 namespace qf {
 
-constexpr int kFuseUnitsPerCta = 16;   // a sweep of at most this many stage units per CTA (bound) is "small"
+constexpr int kSmallUnitsPerCta = 16;   // a sweep of at most this many stage units per CTA (bound) is "small"
 constexpr int kSmallMaxShards  = 32;   // shard slots per request this kernel plans in shared memory
 
 // Can this sweep be treated as small?  Decided on the host from an upper bound on the stage units: every shard of
@@ -38,7 +38,7 @@ inline bool sweep_is_small(const DevParams &P, int n_ctas)
     if (entries > kMaxSmemEntries || P.max_shards > kSmallMaxShards) return false;
     const long long pages = ((long long)P.max_tokens + kPageSize - 1) / kPageSize;
     const long long units = entries * P.num_kv_heads * ((pages + kPagesPerStage - 1) / kPagesPerStage);
-    return units <= (long long)kFuseUnitsPerCta * n_ctas;
+    return units <= (long long)kSmallUnitsPerCta * n_ctas;
 }
 
 // Roles of a CTA, by blockIdx = ((b * Hkv) + c) * (S + 1) + j:

@@ -42,8 +42,8 @@ KERNELS = [pytest.param((0, 16), id="unit16"), pytest.param((0, 8), id="unit8"),
            pytest.param((qf.QF_FLAG_KV_NHD | qf.QF_FLAG_SIMPLE_KERNEL, 2), id="simple-nhd"),
            pytest.param((qf.QF_FLAG_KV_NHD | qf.QF_FLAG_DRAW_ALWAYS, 8), id="draw8-nhd"),
            # a whole step over a small sweep merges with one kernel by default; these keep the finish and merge kernels
-           pytest.param((qf.QF_FLAG_NO_FUSE, 8), id="nofuse8"), pytest.param((qf.QF_FLAG_NO_FUSE, 2), id="nofuse2"),
-           pytest.param((qf.QF_FLAG_NO_FUSE | qf.QF_FLAG_DRAW_ALWAYS, 8), id="nofuse-draw8")]
+           pytest.param((qf.QF_FLAG_NO_SMALL_MERGE, 8), id="nosmall8"), pytest.param((qf.QF_FLAG_NO_SMALL_MERGE, 2), id="nosmall2"),
+           pytest.param((qf.QF_FLAG_NO_SMALL_MERGE | qf.QF_FLAG_DRAW_ALWAYS, 8), id="nosmall-draw8")]
 
 
 # T1: every short length, both group sizes, shuffled table: tail-page masking, first-tile guard
@@ -608,7 +608,7 @@ def test_small_sweeps_merge_with_one_kernel(Hkv, G):
                 assert np.array_equal(x, y)
         # the same as two calls, and as one call with the small path switched off: three kernels, same results
         # within fp32 summation order
-        for dw3 in (run(w, two_calls=True), run(w, qf.QF_FLAG_NO_FUSE)):
+        for dw3 in (run(w, two_calls=True), run(w, qf.QF_FLAG_NO_SMALL_MERGE)):
             assert qf.last_launch_count() in (1, 3)      # the merge alone, or sweep + finish + merge
             T.compare_all(dw3, w)
             for x, y in zip(dw.results(), dw3.results()):
