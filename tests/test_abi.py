@@ -127,3 +127,12 @@ def test_static_scratch_entry_rejects_without_touching_a_device():
     assert qf.decode_partial_static(a, a, a, None, a, a, a, a, a, p, stream=0, check=False) == qf.QF_ERR_BAD_SHAPE
     big = qf.params(batch=4096, num_q_heads=32, num_kv_heads=8, max_pages_per_req=64, max_shards=8, num_pages=1 << 18)
     assert qf.decode_partial_static(a, a, a, None, a, a, a, a, a, big, stream=0, check=False) == qf.QF_ERR_STATIC_SCRATCH
+
+
+def test_peer_access_call_needs_a_device():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    assert qf.enable_peer_access(0, check=False) in (qf.QF_ERR_CUDA, qf.QF_ERR_DEVICE)
+    with pytest.raises(qf.QFError):
+        qf.enable_peer_access(1)
