@@ -119,7 +119,8 @@ __device__ __forceinline__ unsigned epoch_arrive(unsigned long long *w, unsigned
 // a captured CUDA graph distinct (a replay re-runs the kernel with the captured host tag).  The pair is
 // kept as two fields, not a sum, so that an old graph replayed after newer calls cannot land on an
 // epoch a newer call used.  One thread per CTA reads the count at the CTA's start (the caller shares it
-// through shared memory); the CTA that finishes last (epoch-tagged done counter) bumps it for the next launch.
+// through shared memory); the CTA that is the last to have issued all of its work (epoch-tagged done counter: by
+// then every CTA of the launch has read the count) bumps it for the next launch.
 __device__ __forceinline__ unsigned long long launch_epoch(const unsigned long long *header,
                                                            unsigned long long host_epoch)
 {

@@ -478,6 +478,11 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             piece = n_ctas + ticket;
         }
         if (ok) {  // end-of-work marker
+            // This CTA has issued all of its work: count it now, while the consumer warps finish, so that the
+            // arrival's round trips to L2 are off the CTA's exit.  The count only says that every CTA of the
+            // launch has started (each read the launch's epoch before its plan), which is all the last arriver
+            // needs to know before it bumps the launch count for the NEXT launch.
+            if (lane == 0) launch_done(header, epoch, gridDim.x);
             if (mbar_wait(smem_u32(&sm.empty_bar[stage]), phase ^ 1, abort_flag)) {
                 if (lane == 0) {
                     StageMeta mt = {};
@@ -544,10 +549,7 @@ sweep_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ 
             return;
         }
         const StageMeta mt = sm.meta[stage];
-        if (mt.entry < 0) {   // end of this CTA's work
-            if (tid == 0) launch_done(header, epoch, gridDim.x);
-            return;
-        }
+        if (mt.entry < 0) return;   // end of this CTA's work (the producer warp has counted the CTA as done)
 
         if (mt.flags & kSegFirst) {
             const uint16_t *qs = sm.q[stage];
