@@ -47,6 +47,12 @@ def test_one_rank_runs_the_whole_step(transport):
         assert dw.status() == 0
 
 
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
 class _OneProcess:
     """Stands in for the process group when the ranks of a split run one after another in one process."""
     def broadcast(self, t, src=0):
@@ -110,12 +116,59 @@ def test_peer_access_call_on_the_same_device_is_a_no_op():
     assert qf.enable_peer_access(-1, check=False) == qf.QF_ERR_BAD_SHAPE
 
 
-# ---- real ranks, one per GPU (needs at least two)
-def _free_port():
-    with socket.socket() as s:
-        s.bind(("127.0.0.1", 0))
-        return s.getsockname()[1]
+# ---- two PROCESSES on one GPU: everything of the real multi-rank path except NCCL and the cross-device hop.  The
+# owner's arrays travel as CUDA IPC handles over the process group (gloo here) and are opened by the other process,
+# whose sweep stores its shard states into them; no kernel of one process waits for a kernel of the other (the ranks
+# meet in host-side collectives only), so sharing the GPU between the two is safe.
+def _shared_gpu_rank(rank, world, port, out_dir):
+    import datetime
+    import torch.distributed as dist
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    dist.init_process_group("gloo", rank=rank, world_size=world, timeout=datetime.timedelta(seconds=120))
+    try:
+        for i, w in enumerate(workloads()):
+            plan = SplitPlan(world, rank, w.max_shards)
+            runner, out, lse, dw = cuda_runner(w, plan, dist, dev, transport="parked")
+            if rank != plan.owner:
+                dw.q.zero_()                      # only the owner holds the query: it must arrive by broadcast
+                assert runner.owner_arrays[0].data_ptr() != 0
+            for _ in range(3):
+                runner.step()
+            torch.cuda.synchronize()
+            dist.barrier()
+            assert dw.status() == 0
+            if rank == plan.owner:
+                np.save(os.path.join(out_dir, f"out{i}.npy"), out.cpu().numpy())
+                np.save(os.path.join(out_dir, f"lse{i}.npy"), lse.cpu().numpy())
+                np.save(os.path.join(out_dir, f"lpart{i}.npy"), runner.owner_arrays[2].cpu().numpy())
+            dist.barrier()
+            del runner
+    finally:
+        dist.destroy_process_group()
 
+
+def test_two_processes_share_one_gpu_and_the_owners_arrays(tmp_path):
+    import torch.multiprocessing as mp
+    world = 2
+    mp.spawn(_shared_gpu_rank, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    for i, w in enumerate(workloads()):
+        sh = T.oracle_shape(w)
+        ref_out, ref_lse = orc.decode_full(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, sh)
+        assert T.out_err(np.load(tmp_path / f"out{i}.npy"), ref_out) <= T.ENG_OUT
+        assert T.lse_err(np.load(tmp_path / f"lse{i}.npy"), ref_lse) <= T.ENG_LSE
+        # the other process's slots of the owner's arrays hold its shards' states
+        ref_o, ref_m, ref_l = orc.decode_partial(w.q, w.k_cache, w.v_cache, w.block_table, w.seq_lens, w.shard_ranges, sh)
+        got_l = np.load(tmp_path / f"lpart{i}.npy").astype(np.float64)
+        for r in range(world):
+            p = SplitPlan(world, r, w.max_shards)
+            sl = p.slots()
+            assert T.lse_err(got_l[:, p.out_offset:p.out_offset + len(sl)], ref_l[:, sl.start:sl.stop]) <= T.ENG_LSE
+
+
+# ---- real ranks, one per GPU (needs at least two)
 
 def _gpu_rank(rank, world, port, transport, out_dir):
     import torch.distributed as dist
