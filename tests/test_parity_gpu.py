@@ -672,3 +672,35 @@ def test_pipelined_host_steps_match_the_device_path(depth):
     ref = T.oracle_all(w)
     assert T.out_err(got[tickets[-1]][0], ref[3]) <= T.ENG_OUT and T.lse_err(got[tickets[-1]][1], ref[4]) <= T.ENG_LSE
     pipe.close()
+
+
+@pytest.mark.parametrize("seed", list(range(24)))
+def test_randomized_small_steps(seed):
+    # whole steps over small random problems: up to 32 shard slots, random shard counts (0 included), random ranges,
+    # every group size and layout flag; most of them take the one-kernel merge after the sweep
+    rng = np.random.default_rng(5000 + seed)
+    Hkv = int(rng.choice([1, 2, 4, 8, 16]))
+    G = int(rng.integers(1, 9))
+    B = int(rng.integers(1, 13))
+    S = int(rng.choice([1, 2, 3, 5, 8, 13, 32]))
+    maxlen = int(rng.choice([40, 300, 1500, 5000]))
+    lens = [int(x) for x in rng.integers(0, maxlen + 1, size=B)]
+    ranges = []
+    for L in lens:
+        kind = rng.integers(3)
+        if kind == 0:
+            rr = wl.even_shards(L, S)
+        elif kind == 1:
+            rr = wl.fixed_shards(L, max(1, int(rng.integers(1, maxlen + 2))))[:S]
+        else:
+            rr = [tuple(sorted(int(x) for x in rng.integers(-3, L + 5, size=2))) for _ in range(S)]
+        rr = list(rr) + [(0, 0)] * (S - len(rr))
+        ranges.append(rr[:S])
+    counts = [int(rng.integers(0, S + 1)) for _ in lens] if rng.integers(2) else None
+    flags = int(rng.choice([0, qf.QF_FLAG_DRAW_ALWAYS, qf.QF_FLAG_CHECK_BOUNDS, qf.QF_FLAG_KV_NHD]))
+    w = wl.make_workload("small-fuzz", lens, ranges, Hkv * G, Hkv, seed=seed, pool_factor=float(rng.choice([1.0, 1.4])),
+                         poison_unused=True, poison_tails=True, shard_counts=counts,
+                         max_pages_per_req=max(1, (max(lens) + 15) // 16 + int(rng.integers(0, 3))))
+    dw = run(w, flags)
+    T.compare_all(dw, w, tag=f"seed={seed} Hkv={Hkv} G={G} B={B} S={S} flags={flags} launches={qf.last_launch_count()}")
+    assert dw.status() == 0
