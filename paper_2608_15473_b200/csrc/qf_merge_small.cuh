@@ -27,7 +27,10 @@
 
 namespace qf {
 
-constexpr int kSmallUnitsPerCta = 16;   // a sweep of at most this many stage units per CTA (bound) is "small"
+#ifndef QF_SMALL_UNITS_PER_CTA
+#define QF_SMALL_UNITS_PER_CTA 16
+#endif
+constexpr int kSmallUnitsPerCta = QF_SMALL_UNITS_PER_CTA;   // a sweep of at most this many stage units per CTA (bound) is "small"
 constexpr int kSmallMaxShards  = 32;   // shard slots per request this kernel plans in shared memory
 
 // Can this sweep be treated as small?  Decided on the host from an upper bound on the stage units: every shard of
