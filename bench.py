@@ -45,7 +45,7 @@ if str(ROOT) not in sys.path:
 METRIC = "decode-attention KV GB/s and % of B200 HBM peak (Qwen3-4B shape, batched)"
 # dram__bytes_read.sum + dram__bytes_write.sum of one sweep-kernel launch, from the committed ncu summaries
 # (seed 0; see profiles/)
-NCU_TRAFFIC_BYTES = {3: 2013176000 + 5907456, 4: 4295357184 + 508416, 2: 1208430080 + 2514688, 5: 8382518784 + 7926272}
+NCU_TRAFFIC_BYTES = {3: 2013157000 + 5919744, 4: 4295357184 + 508416, 2: 1208430080 + 2514688, 5: 8382518784 + 7926272}
 FALLBACK_HBM_GBS = 6650.0
 DATASHEET_HBM_GBS = 8000.0
 TARGET_LOAD_MS = 400.0       # the timed region of a workload lasts about this long (R repeats of K steps)
